@@ -1,0 +1,489 @@
+// CPU oracle for KV-cache-constrained request scheduling -- TEST INFRASTRUCTURE ONLY.
+//
+// A plain, slow, single-threaded restatement of what the paper defines: the memory model and
+// total end-to-end latency (Section 2.1-2.2, integer program of Section 6.1), the F-metric and
+// Sorted-F (Section 3, Algorithm 1), the exact dynamic programme (Section 5.1, Algorithm 2), and
+// an order-level local search that scores every neighbour with Algorithm 1's Phase 2.  It exists
+// so that the GPU library can be checked against it; it shares no code with that library, is never
+// called by it, and nothing here is tuned for speed.  All arithmetic is integer.
+//
+// Time convention (the paper prints three slightly different ones; this is the integer
+// program's): a request that STARTS at p >= 0 is resident in rounds p+1 .. p+o, uses s + (tau - p)
+// tokens of KV memory in round tau, and COMPLETES at c = p + o.  Algorithm 1's "tentatively set
+// p_i <- t" is therefore read as p_i <- t - 1; with that, its filter p_j + o_j >= t keeps exactly the
+// requests still resident in round t, and the worked example of Section 3 gives 64 and 45.
+//
+// Parity status: every function below is pinned by tests that do not go through this file's own
+// formulas (paper's worked example, closed forms, brute force), except where marked
+// "parity unpinned".
+#include <algorithm>
+#include <cstdint>
+#include <cstring>
+#include <numeric>
+#include <vector>
+
+typedef long long i64;
+typedef unsigned __int128 u128;
+
+extern "C" {
+
+// ---------------------------------------------------------------------------------------------
+// O1. Schedule checker: the integer program's memory row and objective, written out.
+//     Section 6.1: objective  sum_i (start_i + o_i);  memory row for round t:
+//     sum_i sum_{k = max(0, t - o_i)}^{t-1} (s_i + t - k) x_{i,k} <= M.
+// Returns 1 if feasible, 0 if some round exceeds M, -1 on a negative start.
+// ---------------------------------------------------------------------------------------------
+int orc_check_schedule(int n, const int* s, const int* o, i64 M, const i64* p,
+                       i64* tel, i64* peak, i64* first_bad_round, i64* makespan) {
+    i64 horizon = 0;
+    for (int i = 0; i < n; ++i) {
+        if (p[i] < 0) return -1;
+        horizon = std::max(horizon, p[i] + o[i]);
+    }
+    std::vector<i64> U(horizon + 2, 0);                 // U[tau], rounds 1..horizon
+    for (int i = 0; i < n; ++i)
+        for (int j = 1; j <= o[i]; ++j) U[p[i] + j] += (i64)s[i] + j;
+    i64 pk = 0, bad = -1, total = 0;
+    for (i64 tau = 1; tau <= horizon; ++tau) {
+        pk = std::max(pk, U[tau]);
+        if (U[tau] > M && bad < 0) bad = tau;
+    }
+    for (int i = 0; i < n; ++i) total += p[i] + o[i];
+    if (tel) *tel = total;
+    if (peak) *peak = pk;
+    if (first_bad_round) *first_bad_round = bad;
+    if (makespan) *makespan = horizon;
+    return bad < 0 ? 1 : 0;
+}
+
+// Occupancy profile U[tau] for tau = 0..len-1 (U[0] = 0), for tests of "every request decodes
+// exactly o_i tokens" and "occupancy never exceeds M".
+void orc_occupancy(int n, const int* s, const int* o, const i64* p, i64 len, i64* U, i64* resident) {
+    for (i64 t = 0; t < len; ++t) { U[t] = 0; if (resident) resident[t] = 0; }
+    for (int i = 0; i < n; ++i)
+        for (int j = 1; j <= o[i]; ++j)
+            if (p[i] + j < len) { U[p[i] + j] += (i64)s[i] + j; if (resident) resident[p[i] + j] += 1; }
+}
+
+// ---------------------------------------------------------------------------------------------
+// O2. Algorithm 1, Phase 2 ("Scheduling Execution"), step by step.
+//     Each round: t <- t+1; drop completed requests from V; walk the pending list in order; a
+//     request is admitted if, with it added, the memory M(C, e_j) of the combined set C stays
+//     within M at the completion time e_j = p_j + o_j of every member j (Section 3's M(X, t*));
+//     the first request that does not fit ends the round's admissions (break).
+// ---------------------------------------------------------------------------------------------
+static i64 set_memory_at(const std::vector<int>& C, const int* s, const int* o, const i64* p, i64 tstar) {
+    i64 tot = 0;
+    for (int k : C)
+        if ((i64)o[k] >= tstar - p[k]) tot += (i64)s[k] + tstar - p[k];
+    return tot;
+}
+
+int orc_list_schedule_alg1(int n, const int* s, const int* o, i64 M, const int* order,
+                           i64* p, i64* tel, i64* makespan) {
+    for (int i = 0; i < n; ++i)
+        if (s[i] < 1 || o[i] < 1 || (i64)s[i] + o[i] > M) return -1;   // would never be admitted
+    std::vector<int> V;
+    int next = 0;
+    i64 t = 0, last_completion = 0;
+    while (next < n || !V.empty()) {
+        t += 1;
+        std::vector<int> keep;
+        for (int j : V) if (p[j] + o[j] >= t) keep.push_back(j);
+        V.swap(keep);
+        while (next < n) {
+            int i = order[next];
+            p[i] = t - 1;                               // starts now: first resident round is t
+            std::vector<int> C(V);
+            C.push_back(i);
+            bool ok = true;
+            for (int j : C)
+                if (set_memory_at(C, s, o, p, p[j] + o[j]) > M) { ok = false; break; }
+            if (!ok) break;
+            V.swap(C);
+            last_completion = std::max(last_completion, p[i] + o[i]);
+            ++next;
+        }
+    }
+    i64 total = 0;
+    for (int i = 0; i < n; ++i) total += p[i] + o[i];
+    if (tel) *tel = total;
+    if (makespan) *makespan = last_completion;
+    return 0;
+}
+
+// O2'. The same executor stated on the per-round occupancy array instead of on completion times:
+//      a request fits at start k iff U[k+j] + s + j <= M for every j = 1..o (Section 2.1's batch
+//      memory constraint in every round it is resident); if not, it is retried one round later and
+//      nothing behind it is looked at (the break).  Used where O2's quadratic set test is too slow;
+//      tests check O2 == O2' on many instances.
+int orc_list_schedule_rounds(int n, const int* s, const int* o, i64 M, const int* order,
+                             i64* p, i64* tel, i64* makespan) {
+    i64 sum_o = 0; int omax = 0;
+    for (int i = 0; i < n; ++i) {
+        if (s[i] < 1 || o[i] < 1 || (i64)s[i] + o[i] > M) return -1;
+        sum_o += o[i]; omax = std::max(omax, o[i]);
+    }
+    std::vector<i64> U(sum_o + omax + 2, 0);
+    i64 k = 0, total = 0, last = 0;
+    for (int q = 0; q < n; ++q) {
+        int i = order[q];
+        for (;;) {
+            bool fits = true;
+            for (int j = 1; j <= o[i]; ++j)
+                if (U[k + j] + s[i] + j > M) { fits = false; break; }
+            if (fits) break;
+            k += 1;
+        }
+        p[i] = k;
+        for (int j = 1; j <= o[i]; ++j) U[k + j] += (i64)s[i] + j;
+        total += k + o[i];
+        last = std::max(last, k + o[i]);
+    }
+    if (tel) *tel = total;
+    if (makespan) *makespan = last;
+    return 0;
+}
+
+// ---------------------------------------------------------------------------------------------
+// O3. Order policies.  0 = FCFS (index order, Section 7), 1 = shortest output first (MC-SF,
+//     Section 2.3), 2 = smallest s+o first (MC-SF_2, Appendix A).  Ties: lower index first.
+// ---------------------------------------------------------------------------------------------
+void orc_policy_order(int n, const int* s, const int* o, int policy, int* order) {
+    std::iota(order, order + n, 0);
+    if (policy == 1)
+        std::stable_sort(order, order + n, [&](int a, int b) { return o[a] < o[b]; });
+    else if (policy == 2)
+        std::stable_sort(order, order + n, [&](int a, int b) { return s[a] + o[a] < s[b] + o[b]; });
+}
+
+// ---------------------------------------------------------------------------------------------
+// F-metric comparison (Section 3): F(X) = sum_o / |X|^2, smaller first, ties -> larger batch.
+// Exact: sumA / kA^2 < sumB / kB^2  <=>  sumA * kB^2 < sumB * kA^2.
+// Returns <0 if A is better, >0 if B is better, 0 if (F, |X|) are equal.
+// ---------------------------------------------------------------------------------------------
+int orc_f_compare(i64 sumA, i64 kA, i64 sumB, i64 kB) {
+    u128 l = (u128)sumA * (u128)kB * (u128)kB, r = (u128)sumB * (u128)kA * (u128)kA;
+    if (l != r) return l < r ? -1 : 1;
+    if (kA != kB) return kA > kB ? -1 : 1;
+    return 0;
+}
+
+// ---------------------------------------------------------------------------------------------
+// O4. Exact Phase 1 by enumeration of all non-empty subsets of `ids` (m <= 24).
+//     reading 0: Algorithm 1's constraint  M(X, o_j) <= M for all j in X  with all of X started
+//                together, i.e. sum_{i in X, o_i >= o_j} (s_i + o_j) <= M;
+//     reading 1: sum (s_i + o_i) <= M, the constraint Algorithms 2, 4 and 5 use.
+//     Minimise (F, -|X|); then smaller sum(s+o); then the lexicographically smallest index list.
+// Writes the chosen members (ascending position in `ids`) and returns their count.
+// ---------------------------------------------------------------------------------------------
+int orc_phase1_enumerate(int m, const int* ids, const int* s, const int* o, i64 M, int reading,
+                         int* chosen, i64* sum_o_out, i64* mem_out) {
+    if (m > 24) return -1;
+    i64 bestSum = 0, bestMem = 0; int bestK = 0; unsigned bestMask = 0;
+    for (unsigned mask = 1; mask < (1u << m); ++mask) {
+        i64 so = 0, mem = 0; int k = 0;
+        for (int a = 0; a < m; ++a) if (mask >> a & 1) { so += o[ids[a]]; mem += s[ids[a]] + o[ids[a]]; ++k; }
+        bool feas;
+        if (reading == 1) feas = mem <= M;
+        else {
+            feas = true;
+            for (int a = 0; a < m && feas; ++a) if (mask >> a & 1) {
+                i64 tot = 0;
+                for (int b = 0; b < m; ++b)
+                    if ((mask >> b & 1) && o[ids[b]] >= o[ids[a]]) tot += (i64)s[ids[b]] + o[ids[a]];
+                if (tot > M) feas = false;
+            }
+        }
+        if (!feas) continue;
+        bool better;
+        if (bestK == 0) better = true;
+        else {
+            int c = orc_f_compare(so, k, bestSum, bestK);
+            if (c != 0) better = c < 0;
+            else if (mem != bestMem) better = mem < bestMem;
+            else {
+                // same size: the list with the smaller first differing member wins
+                unsigned diff = mask ^ bestMask;
+                unsigned low = diff & (~diff + 1);
+                better = (mask & low) != 0;
+            }
+        }
+        if (better) { bestSum = so; bestMem = mem; bestK = k; bestMask = mask; }
+    }
+    int c = 0;
+    for (int a = 0; a < m; ++a) if (bestMask >> a & 1) chosen[c++] = ids[a];
+    if (sum_o_out) *sum_o_out = bestSum;
+    if (mem_out) *mem_out = bestMem;
+    return c;
+}
+
+// ---------------------------------------------------------------------------------------------
+// O5. Algorithm 2 (exact dynamic programme), as printed: dp[k][m] = min sum of o over k-subsets
+//     whose sum(s+o) is exactly m; requests taken one at a time, k descending, strict '<' update;
+//     path[k][m] kept as a bit set (m <= 128 requests).  The final scan follows Section 3's tie
+//     rule (min F, then larger k, then smaller m) rather than the listing's first-strictly-smaller
+//     scan, because the analysis relies on "ties -> larger batch".
+// ---------------------------------------------------------------------------------------------
+int orc_phase1_dp(int m, const int* ids, const int* s, const int* o, i64 M,
+                  int* chosen, i64* sum_o_out, i64* mem_out) {
+    if (m > 128 || M > (1 << 22)) return -1;
+    const i64 INF = INT64_MAX;
+    const int W = (int)M + 1;
+    std::vector<i64> dp((size_t)(m + 1) * W, INF);
+    struct Bits { uint64_t w[2]; };
+    std::vector<Bits> path((size_t)(m + 1) * W, Bits{{0, 0}});
+    dp[0] = 0;
+    for (int a = 0; a < m; ++a) {
+        int mi = s[ids[a]] + o[ids[a]], oi = o[ids[a]];
+        for (int k = a; k >= 0; --k)                    // k <= a: at most a requests seen so far
+            for (int mm = 0; mm + mi <= M; ++mm) {
+                i64 cur = dp[(size_t)k * W + mm];
+                if (cur == INF) continue;
+                i64 nv = cur + oi;
+                size_t dst = (size_t)(k + 1) * W + mm + mi;
+                if (nv < dp[dst]) {
+                    dp[dst] = nv;
+                    path[dst] = path[(size_t)k * W + mm];
+                    path[dst].w[a >> 6] |= 1ull << (a & 63);
+                }
+            }
+    }
+    int bestK = 0; i64 bestSum = 0; int bestM = 0;
+    for (int k = 1; k <= m; ++k)
+        for (int mm = 0; mm <= M; ++mm) {
+            i64 v = dp[(size_t)k * W + mm];
+            if (v == INF) continue;
+            bool better = bestK == 0;
+            if (!better) {
+                int c = orc_f_compare(v, k, bestSum, bestK);
+                better = c < 0;                          // equal (F, k): the smaller m was seen first
+            }
+            if (better) { bestK = k; bestSum = v; bestM = mm; }
+        }
+    const Bits& b = path[(size_t)bestK * W + bestM];
+    int c = 0;
+    for (int a = 0; a < m; ++a) if (b.w[a >> 6] >> (a & 63) & 1) chosen[c++] = ids[a];
+    if (sum_o_out) *sum_o_out = bestSum;
+    if (mem_out) *mem_out = bestM;
+    return c;
+}
+
+// ---------------------------------------------------------------------------------------------
+// O7. Sorted-F assembly (Algorithm 1, Phase 1 loop) around a Phase-1 solver:
+//     solver 0 = enumeration with Algorithm 1's own constraint, 1 = enumeration with sum(s+o)<=M,
+//     2 = Algorithm 2.  Each selected batch is sorted by nondecreasing o (ties: lower index) and
+//     appended.  batch_offsets gets num_batches+1 entries.
+// ---------------------------------------------------------------------------------------------
+int orc_sorted_f_exact(int n, const int* s, const int* o, i64 M, int solver,
+                       int* order, int* batch_offsets) {
+    std::vector<int> rem(n);
+    std::iota(rem.begin(), rem.end(), 0);
+    int pos = 0, nb = 0;
+    batch_offsets[0] = 0;
+    std::vector<int> chosen(n);
+    while (!rem.empty()) {
+        int c;
+        if (solver == 2) c = orc_phase1_dp((int)rem.size(), rem.data(), s, o, M, chosen.data(), 0, 0);
+        else c = orc_phase1_enumerate((int)rem.size(), rem.data(), s, o, M, solver, chosen.data(), 0, 0);
+        if (c <= 0) return -1;
+        std::vector<int> X(chosen.begin(), chosen.begin() + c);
+        std::stable_sort(X.begin(), X.end(), [&](int a, int b) { return o[a] < o[b]; });
+        for (int x : X) order[pos++] = x;
+        batch_offsets[++nb] = pos;
+        std::vector<int> rest;
+        for (int r : rem) if (std::find(chosen.begin(), chosen.begin() + c, r) == chosen.begin() + c) rest.push_back(r);
+        rem.swap(rest);
+    }
+    return nb;
+}
+
+// ---------------------------------------------------------------------------------------------
+// O6. Prefix-F batch selection -- a scalable stand-in for Algorithm 1's argmin that the paper does
+//     not print: candidates are restricted to prefixes of the remaining requests in the order
+//     Algorithm 4 starts from (ascending s+o; ties by o, then index).  From offset a, with
+//     k_max the longest prefix whose sum(s+o) <= M, pick k minimising (F, -k) over 1..k_max,
+//     append that prefix sorted by (o, index), continue from a + k.
+// ---------------------------------------------------------------------------------------------
+int orc_sorted_f_prefix(int n, const int* s, const int* o, i64 M, int* order, int* batch_offsets) {
+    std::vector<int> idx(n);
+    std::iota(idx.begin(), idx.end(), 0);
+    std::stable_sort(idx.begin(), idx.end(), [&](int a, int b) {
+        int ta = s[a] + o[a], tb = s[b] + o[b];
+        if (ta != tb) return ta < tb;
+        return o[a] < o[b];
+    });
+    int a = 0, nb = 0;
+    batch_offsets[0] = 0;
+    while (a < n) {
+        i64 mem = 0, so = 0, bestSum = 0; int bestK = 0;
+        for (int k = 1; a + k <= n; ++k) {
+            int r = idx[a + k - 1];
+            mem += s[r] + o[r];
+            if (mem > M) break;
+            so += o[r];
+            if (bestK == 0 || orc_f_compare(so, k, bestSum, bestK) < 0) { bestK = k; bestSum = so; }
+        }
+        if (bestK == 0) return -1;                       // a single request exceeds M
+        std::vector<int> X(idx.begin() + a, idx.begin() + a + bestK);
+        std::stable_sort(X.begin(), X.end(), [&](int x, int y) {
+            if (o[x] != o[y]) return o[x] < o[y];
+            return x < y;
+        });
+        for (int k = 0; k < bestK; ++k) order[a + k] = X[k];
+        a += bestK;
+        batch_offsets[++nb] = a;
+    }
+    return nb;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Moves on an order (used by the local search; the paper's swap idea of Section 5.2 applied to
+// positions of the ordered list).  Codes: swaps (i, j), 0 <= i < j < n, in lexicographic order,
+// codes 0 .. n(n-1)/2 - 1; then inserts (i -> j), i != j: take the request at position i out and
+// put it back so that it sits at position j, code n(n-1)/2 + i (n-1) + (j < i ? j : j - 1).
+// ---------------------------------------------------------------------------------------------
+int orc_decode_move(int n, i64 code, int* type, int* i_out, int* j_out) {
+    i64 nsw = (i64)n * (n - 1) / 2;
+    if (code < 0 || code >= nsw + (i64)n * (n - 1)) return -1;
+    if (code < nsw) {
+        int i = 0; i64 c = code;
+        while (c >= n - 1 - i) { c -= n - 1 - i; ++i; }
+        *type = 0; *i_out = i; *j_out = i + 1 + (int)c;
+    } else {
+        i64 c = code - nsw;
+        int i = (int)(c / (n - 1)), r = (int)(c % (n - 1));
+        *type = 1; *i_out = i; *j_out = r < i ? r : r + 1;
+    }
+    return 0;
+}
+
+void orc_apply_move(int n, const int* base, int type, int i, int j, int* out) {
+    std::vector<int> v(base, base + n);
+    if (type == 0) std::swap(v[i], v[j]);
+    else { int x = v[i]; v.erase(v.begin() + i); v.insert(v.begin() + j, x); }
+    std::copy(v.begin(), v.end(), out);
+}
+
+// splitmix64 finaliser; the sampled neighbourhood derives move m of iteration it from
+// h1 = mix(seed ^ mix(it * 2^32 + m)), h2 = mix(h1): type = h1 & 1, i = (h1 >> 1) mod n,
+// j = (i + 1 + h2 mod (n-1)) mod n; a swap is normalised to i < j.
+static uint64_t mix64(uint64_t z) {
+    z += 0x9E3779B97F4A7C15ull;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
+}
+
+void orc_sample_move(int n, uint64_t seed, int it, i64 m, int* type, int* i_out, int* j_out) {
+    uint64_t h1 = mix64(seed ^ mix64(((uint64_t)(uint32_t)it << 32) + (uint64_t)m));
+    uint64_t h2 = mix64(h1);
+    int ty = (int)(h1 & 1);
+    int i = (int)((h1 >> 1) % (uint64_t)n);
+    int j = (int)(((uint64_t)i + 1 + h2 % (uint64_t)(n - 1)) % (uint64_t)n);
+    if (ty == 0 && i > j) std::swap(i, j);
+    *type = ty; *i_out = i; *j_out = j;
+}
+
+// Evaluate a list of moves against one base order with O2'.
+int orc_eval_moves(int n, const int* s, const int* o, i64 M, const int* base,
+                   i64 count, const int* type, const int* mi, const int* mj, i64* tel_out) {
+    std::vector<int> cand(n);
+    std::vector<i64> p(n);
+    for (i64 c = 0; c < count; ++c) {
+        orc_apply_move(n, base, type[c], mi[c], mj[c], cand.data());
+        if (orc_list_schedule_rounds(n, s, o, M, cand.data(), p.data(), &tel_out[c], 0)) return -1;
+    }
+    return 0;
+}
+
+// ---------------------------------------------------------------------------------------------
+// O8. Order-level local search.  neighbourhood 0 = all swaps, 1 = all swaps then all inserts,
+//     2 = `samples` sampled moves per iteration.  Per iteration: best = min (TEL, code) over the
+//     neighbourhood (code = move code, or the sample index m); accept iff TEL_best < TEL_cur
+//     (strict, as in Section 5.2's improving-swap rule).  Full neighbourhoods stop at a local
+//     optimum; the sampled one always runs `iters` iterations.
+//     trace (nullable) receives, per iteration, (code, TEL_best) -- 2 entries each.
+// ---------------------------------------------------------------------------------------------
+int orc_local_search(int n, const int* s, const int* o, i64 M, int neighbourhood, int iters,
+                     uint64_t seed, i64 samples, int* order, i64* tel_out, int* iters_done, i64* trace) {
+    std::vector<int> cand(n);
+    std::vector<i64> p(n);
+    i64 cur;
+    if (orc_list_schedule_rounds(n, s, o, M, order, p.data(), &cur, 0)) return -1;
+    i64 nsw = (i64)n * (n - 1) / 2;
+    i64 ncodes = neighbourhood == 0 ? nsw : neighbourhood == 1 ? nsw + (i64)n * (n - 1) : samples;
+    int it = 0;
+    for (; it < iters; ++it) {
+        i64 best = INT64_MAX, bestCode = -1; int bt = 0, bi = 0, bj = 0;
+        for (i64 c = 0; c < ncodes; ++c) {
+            int ty, i, j;
+            if (neighbourhood == 2) orc_sample_move(n, seed, it, c, &ty, &i, &j);
+            else orc_decode_move(n, c, &ty, &i, &j);
+            orc_apply_move(n, order, ty, i, j, cand.data());
+            i64 tel;
+            orc_list_schedule_rounds(n, s, o, M, cand.data(), p.data(), &tel, 0);
+            if (tel < best) { best = tel; bestCode = c; bt = ty; bi = i; bj = j; }
+        }
+        if (trace) { trace[2 * it] = bestCode; trace[2 * it + 1] = best; }
+        if (bestCode >= 0 && best < cur) {
+            orc_apply_move(n, order, bt, bi, bj, cand.data());
+            std::copy(cand.begin(), cand.end(), order);
+            cur = best;
+        } else if (neighbourhood != 2) { ++it; break; }
+    }
+    *tel_out = cur;
+    *iters_done = it;
+    return 0;
+}
+
+// ---------------------------------------------------------------------------------------------
+// O9. Brute force for tiny instances.
+//  (i)  True optimum of the integer program: depth-first over start-time vectors, request by
+//       request, every start 0..slack tried, feasibility by the occupancy definition; pruned only
+//       by the objective (sum of starts already above the best known).
+//  (ii) Best list schedule over all n! orders through O2.
+// ---------------------------------------------------------------------------------------------
+struct BF { int n; const int* s; const int* o; i64 M; i64 best; std::vector<i64> U; std::vector<i64> p, bestp; i64 sum_o; };
+
+static void bf_rec(BF& b, int i, i64 sum_p) {
+    if (sum_p + b.sum_o >= b.best) return;
+    if (i == b.n) { b.best = sum_p + b.sum_o; b.bestp = b.p; return; }
+    i64 slack = b.best - 1 - b.sum_o - sum_p;            // largest start that can still improve
+    for (i64 k = 0; k <= slack; ++k) {
+        bool ok = true;
+        for (int j = 1; j <= b.o[i]; ++j) if (b.U[k + j] + b.s[i] + j > b.M) { ok = false; break; }
+        if (!ok) continue;
+        for (int j = 1; j <= b.o[i]; ++j) b.U[k + j] += b.s[i] + j;
+        b.p[i] = k;
+        bf_rec(b, i + 1, sum_p + k);
+        for (int j = 1; j <= b.o[i]; ++j) b.U[k + j] -= b.s[i] + j;
+    }
+}
+
+// upper_bound: any TEL known to be achievable (e.g. a list schedule's) + 1, to bound the search.
+i64 orc_bruteforce_opt(int n, const int* s, const int* o, i64 M, i64 upper_bound, i64* p_out) {
+    BF b; b.n = n; b.s = s; b.o = o; b.M = M; b.best = upper_bound; b.sum_o = 0;
+    int omax = 0;
+    for (int i = 0; i < n; ++i) { b.sum_o += o[i]; omax = std::max(omax, o[i]); }
+    b.U.assign(upper_bound + omax + 2, 0);
+    b.p.assign(n, 0);
+    bf_rec(b, 0, 0);
+    if (p_out && !b.bestp.empty()) for (int i = 0; i < n; ++i) p_out[i] = b.bestp[i];
+    return b.bestp.empty() ? -1 : b.best;
+}
+
+i64 orc_bruteforce_best_order(int n, const int* s, const int* o, i64 M, int* best_order) {
+    std::vector<int> perm(n);
+    std::iota(perm.begin(), perm.end(), 0);
+    std::vector<i64> p(n);
+    i64 best = INT64_MAX;
+    do {
+        i64 tel;
+        if (orc_list_schedule_alg1(n, s, o, M, perm.data(), p.data(), &tel, 0)) return -1;
+        if (tel < best) { best = tel; if (best_order) std::copy(perm.begin(), perm.end(), best_order); }
+    } while (std::next_permutation(perm.begin(), perm.end()));
+    return best;
+}
+
+}  // extern "C"

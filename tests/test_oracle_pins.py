@@ -1,0 +1,411 @@
+"""Pins for the CPU oracle: values the paper prints, closed forms, brute force, invariants.
+
+Each test is chosen so that a plausible slip in the oracle (an off-by-one in the time convention,
+skip instead of break, a dropped ramp term, a transposed comparison, a wrong tie rule) fails it.
+No expected value here comes from the oracle itself or from the GPU library.
+"""
+import itertools
+
+import numpy as np
+import pytest
+
+import oracle as orc
+from paper_2508_06133_b200 import workloads as W
+
+
+# ----------------------------------------------------------------------------- worked example
+def example1():
+    s = np.array([63] + [1] * 21, dtype=np.int32)
+    o = np.array([1] + [2] * 21, dtype=np.int32)
+    return s, o
+
+
+@pytest.mark.parametrize("executor", [orc.list_schedule_alg1, orc.list_schedule_rounds])
+def test_example1_tel(golden, executor):
+    s, o = example1()
+    M = golden["example1_M"]
+    mcsf = orc.policy_order(s, o, orc.SHORTEST_OUTPUT_FIRST)
+    assert mcsf[0] == 0                                   # the o = 1 request goes first
+    assert executor(s, o, M, mcsf)[1] == golden["example1_tel_mcsf"]
+    sorted_f = np.array(list(range(1, 22)) + [0], dtype=np.int32)
+    p, tel, mk = executor(s, o, M, sorted_f)
+    assert tel == golden["example1_tel_sortedf"]
+    assert mk == 3 and p[0] == 2 and (p[1:] == 0).all()   # Type 2 done at t=2, Type 1 runs in round 3
+
+
+def test_example1_checker_by_hand(golden):
+    """Start vectors written by hand, checked by the occupancy definition."""
+    s, o = example1()
+    M = golden["example1_M"]
+    good = np.array([2] + [0] * 21)
+    r = orc.check_schedule(s, o, M, good)
+    assert r["feasible"] and r["tel"] == 45 and r["peak"] == 64 and r["makespan"] == 3
+    bad = np.array([1] + [0] * 21)                         # Type 1 overlaps the round where Type 2 holds 63
+    r = orc.check_schedule(s, o, M, bad)
+    assert not r["feasible"] and r["first_bad_round"] == 2 and r["peak"] == 63 + 64
+    # 22 Type-2 requests together need 66 > 64 in their second round: capacity is 21
+    s22, o22 = np.ones(22, dtype=np.int32), np.full(22, 2, dtype=np.int32)
+    assert not orc.check_schedule(s22, o22, M, np.zeros(22))["feasible"]
+    assert orc.check_schedule(s22[:21], o22[:21], M, np.zeros(21))["feasible"]
+    assert golden["example1_batch_capacity"] == 21
+
+
+def test_example1_f_metric(golden):
+    # F(Type 2 x 21) = 42/441 < F(Type 1) = 1/1
+    assert orc.f_compare(golden["example1_F_type2_num"], 21, golden["example1_F_type1_num"], 1) < 0
+    assert orc.f_compare(1, 1, 42, 21) > 0
+    assert golden["example1_F_type2_den"] == 21 ** 2
+    # ties on F prefer the larger batch: 2/2^2 == 8/4^2
+    assert orc.f_compare(8, 4, 2, 2) < 0 and orc.f_compare(2, 2, 8, 4) > 0 and orc.f_compare(3, 3, 3, 3) == 0
+    # products beyond 64 bits still compare exactly
+    assert orc.f_compare(4 * 10 ** 8, 10 ** 5, 4 * 10 ** 8 + 1, 10 ** 5) < 0
+
+
+def test_example1_sorted_f_selects_type2_first(golden):
+    s, o = example1()
+    M = golden["example1_M"]
+    for solver in (orc.ENUM_SUM, orc.DP):
+        ids = np.arange(22)
+        chosen, so, mem = (orc.phase1_enumerate(ids[:14], s, o, M, solver) if solver != orc.DP
+                           else orc.phase1_dp(ids, s, o, M))
+        assert 0 not in chosen                            # never the prompt-63 request
+    order, offs = orc.sorted_f_exact(s, o, M, orc.DP)
+    assert list(offs) == [0, 21, 22] and order[-1] == 0
+    order, offs = orc.sorted_f_prefix(s, o, M)
+    assert list(offs) == [0, 21, 22] and order[-1] == 0
+    assert orc.list_schedule_alg1(s, o, M, order)[1] == golden["example1_tel_sortedf"]
+
+
+# ----------------------------------------------------------------------------- Example 2 (symbolic)
+@pytest.mark.parametrize("n1,s1,o1,n2,s2,o2", [(10, 8, 4, 4, 20, 10), (6, 15, 5, 3, 28, 12), (5, 10, 14, 12, 4, 6)])
+def test_example2_two_saturating_batches(n1, s1, o1, n2, s2, o2):
+    """Appendix B, Example 2: n1(s1+o1) = n2(s2+o2) = M; TEL = o1 n1 + o2 n2 + (o1 n2 | o2 n1)."""
+    M = n1 * (s1 + o1)
+    assert M == n2 * (s2 + o2)
+    s = np.array([s1] * n1 + [s2] * n2, dtype=np.int32)
+    o = np.array([o1] * n1 + [o2] * n2, dtype=np.int32)
+    first1 = np.arange(n1 + n2)
+    first2 = np.concatenate([np.arange(n1, n1 + n2), np.arange(n1)])
+    # The example's totals assume the second batch cannot overlap the first.  Under continuous
+    # batching that holds exactly when the second batch's requests outlive the first batch's
+    # saturated last round (o_second >= o_first); otherwise early starts can only lower the TEL.
+    tel12 = o1 * n1 + o2 * n2 + o1 * n2
+    tel21 = o1 * n1 + o2 * n2 + o2 * n1
+    for ex in (orc.list_schedule_alg1, orc.list_schedule_rounds):
+        got12, got21 = ex(s, o, M, first1)[1], ex(s, o, M, first2)[1]
+        assert got12 == tel12 if o2 >= o1 else got12 <= tel12
+        assert got21 == tel21 if o1 >= o2 else got21 <= tel21
+    # the F rule prefers the order the example says is cheaper
+    prefer1 = orc.f_compare(o1 * n1, n1, o2 * n2, n2) < 0
+    assert prefer1 == (o1 * n2 < o2 * n1)
+
+
+# ----------------------------------------------------------------------------- Theorem 1 closed form
+@pytest.mark.parametrize("root4", [3, 6, 9])
+def test_theorem1_closed_form(root4, golden):
+    """Appendix A: X = M requests (sqrt(M)-1, 1) then Y = M^1.25 requests (1, 2), shortest output first."""
+    M = root4 ** 4
+    r = root4 ** 2
+    X, Y = M, root4 ** 5
+    assert M % 3 == 0
+    s = np.array([r - 1] * X + [1] * Y, dtype=np.int32)
+    o = np.array([1] * X + [2] * Y, dtype=np.int32)
+    order = orc.policy_order(s, o, orc.SHORTEST_OUTPUT_FIRST)
+    assert (order == np.arange(X + Y)).all()
+    tri = lambda k: k * (k + 1) // 2
+    closed = r * tri(X // r) + X * Y // r + (2 * M // 3) * tri(3 * Y // M)
+    if M == 6561:
+        assert closed == golden["thm1_M6561_tel_mcsf"]
+    assert orc.list_schedule_rounds(s, o, M, order)[1] == closed
+    if M <= 1296:
+        assert orc.list_schedule_alg1(s, o, M, order)[1] == closed
+
+
+# ----------------------------------------------------------------------------- NP-hardness family
+def test_three_partition_family(golden):
+    """Appendix A: s_i = x_i, o_i = 1, M = T + 3; optimum 3m(m+1)/2 iff a 3-partition exists."""
+    T = 20
+    x = [6, 7, 7, 6, 6, 8]                                # {6,7,7}, {6,6,8}
+    s, o = np.array(x, dtype=np.int32), np.ones(6, dtype=np.int32)
+    M = T + 3
+    opt, p = orc.bruteforce_opt(s, o, M, 6 * 7)
+    assert opt == golden["np_family_m2"]
+    assert orc.check_schedule(s, o, M, p)["feasible"]
+    assert np.bincount(p.astype(int)).tolist() == [3, 3]
+    # the partition given as an order reaches it through the executor
+    assert orc.list_schedule_alg1(s, o, M, [0, 1, 2, 3, 4, 5])[1] == 9
+    best, _ = orc.bruteforce_best_order(s, o, M)
+    assert best == 9
+    # no batch of four fits
+    for quad in itertools.combinations(range(6), 4):
+        pp = np.array([0 if i in quad else 5 for i in range(6)])
+        assert not orc.check_schedule(s, o, M, pp)["feasible"]
+    # no 3-partition: {6,6,6,6,7,9} has no triple summing to 20
+    x2 = [6, 6, 6, 6, 7, 9]
+    assert sum(x2) == 2 * T and all(sum(c) != T for c in itertools.combinations(x2, 3))
+    opt2, _ = orc.bruteforce_opt(np.array(x2, dtype=np.int32), o, M, 6 * 7)
+    assert opt2 > 9
+    # m = 3
+    x3 = [6, 7, 7, 6, 6, 8, 8, 6, 6]
+    s3, o3 = np.array(x3, dtype=np.int32), np.ones(9, dtype=np.int32)
+    opt3, _ = orc.bruteforce_opt(s3, o3, M, 9 * 10)
+    assert opt3 == golden["np_family_m3"]
+
+
+# ----------------------------------------------------------------------------- executor invariants
+def random_instance(rng, n, M, smax, omax):
+    s = rng.integers(1, smax + 1, n).astype(np.int32)
+    o = rng.integers(1, omax + 1, n).astype(np.int32)
+    keep = s + o <= M
+    s[~keep] = 1
+    return s, o
+
+
+def numpy_occupancy(s, o, p, length):
+    """Independent restatement of the memory model (Section 2.1): token j of request i needs s_i + j."""
+    U = np.zeros(length, dtype=np.int64)
+    for si, oi, pi in zip(s, o, p):
+        U[pi + 1: pi + oi + 1] += si + np.arange(1, oi + 1)
+    return U
+
+
+def test_alg1_equals_round_form_and_invariants():
+    rng = np.random.default_rng(12345)
+    for trial in range(300):
+        n = int(rng.integers(1, 40))
+        M = int(rng.integers(8, 200))
+        s, o = random_instance(rng, n, M, max(1, M // 2), max(1, M // 3))
+        order = rng.permutation(n).astype(np.int32)
+        p1, tel1, mk1 = orc.list_schedule_alg1(s, o, M, order)
+        p2, tel2, mk2 = orc.list_schedule_rounds(s, o, M, order)
+        assert (p1 == p2).all() and tel1 == tel2 and mk1 == mk2
+        assert tel1 == int((p1 + o).sum())
+        chk = orc.check_schedule(s, o, M, p1)
+        assert chk["feasible"] and chk["tel"] == tel1 and chk["peak"] <= M and chk["makespan"] == mk1
+        U = numpy_occupancy(s, o, p1, mk1 + 2)
+        assert U.max() == chk["peak"] <= M
+        Uo, R = orc.occupancy(s, o, p1, mk1 + 2)
+        assert (Uo == U).all() and R.sum() == o.sum()      # every request decodes exactly o_i tokens
+        # starts never go backwards along the order (first misfit blocks everything behind it)
+        assert (np.diff(p1[order]) >= 0).all()
+
+
+def test_each_start_is_the_earliest_feasible():
+    """Break rule + maximal admission: request q starts at the first round >= its predecessor's
+    start at which the occupancy definition admits it, given the earlier requests."""
+    rng = np.random.default_rng(777)
+    for trial in range(60):
+        n = int(rng.integers(2, 14))
+        M = int(rng.integers(10, 80))
+        s, o = random_instance(rng, n, M, M // 2, M // 3 + 1)
+        order = rng.permutation(n)
+        p, tel, mk = orc.list_schedule_alg1(s, o, M, order)
+        for q in range(n):
+            sub = order[:q + 1]
+            lo = p[order[q - 1]] if q else 0
+            for k in range(lo, p[order[q]]):               # every earlier admissible start must overflow
+                pp = p[sub].copy()
+                pp[-1] = k
+                assert not orc.check_schedule(s[sub], o[sub], M, pp)["feasible"]
+            assert orc.check_schedule(s[sub], o[sub], M, p[sub])["feasible"]
+
+
+def test_invalid_instances_rejected():
+    with pytest.raises(ValueError):
+        orc.list_schedule_alg1([5], [6], 10, [0])          # s + o > M would never be admitted
+    with pytest.raises(ValueError):
+        orc.list_schedule_rounds([0], [1], 10, [0])
+    assert orc.check_schedule([1], [1], 10, [-1])["rc"] == -1
+
+
+def test_policies():
+    s = np.array([5, 1, 3, 1, 9], dtype=np.int32)
+    o = np.array([2, 7, 2, 3, 1], dtype=np.int32)
+    assert orc.policy_order(s, o, orc.FCFS).tolist() == [0, 1, 2, 3, 4]
+    assert orc.policy_order(s, o, orc.SHORTEST_OUTPUT_FIRST).tolist() == [4, 0, 2, 3, 1]
+    assert orc.policy_order(s, o, orc.TOTAL_SIZE_FIRST).tolist() == [3, 2, 0, 1, 4]   # sizes 7,8,5,4,10
+
+
+# ----------------------------------------------------------------------------- Phase 1 solvers
+def test_phase1_dp_matches_enumeration_and_lemma1():
+    rng = np.random.default_rng(99)
+    for trial in range(120):
+        n = int(rng.integers(2, 13))
+        M = int(rng.integers(12, 90))
+        s, o = random_instance(rng, n, M, M // 2, M // 2)
+        ids = np.arange(n)
+        ce, so_e, mem_e = orc.phase1_enumerate(ids, s, o, M, orc.ENUM_SUM)
+        cd, so_d, mem_d = orc.phase1_dp(ids, s, o, M)
+        assert (so_e, len(ce), mem_e) == (so_d, len(cd), mem_d)
+        assert int(o[cd].sum()) == so_d and int((s[cd] + o[cd]).sum()) == mem_d <= M
+        # brute force in Python over all subsets: nothing feasible has a smaller (F, -k)
+        for k in range(1, n + 1):
+            for sub in itertools.combinations(range(n), k):
+                sub = list(sub)
+                if int((s[sub] + o[sub]).sum()) <= M:
+                    lhs, rhs = int(o[sub].sum()) * len(cd) ** 2, so_d * k ** 2
+                    assert lhs > rhs or (lhs == rhs and k <= len(cd))
+        # Lemma 1: mean output of an exactly selected batch exceeds half its largest output
+        for chosen in (ce, cd):
+            assert 2 * int(o[chosen].sum()) > int(o[chosen].max()) * len(chosen)
+        # sum(s+o) <= M implies Algorithm 1's own constraint, so its optimum is at least as good
+        ca, so_a, _ = orc.phase1_enumerate(ids, s, o, M, orc.ENUM_ALG1)
+        assert orc.f_compare(so_a, len(ca), so_e, len(ce)) <= 0
+        assert 2 * int(o[ca].sum()) > int(o[ca].max()) * len(ca)
+        # the Algorithm-1 batch really is feasible when started together
+        assert orc.check_schedule(s[ca], o[ca], M, np.zeros(len(ca)))["feasible"]
+
+
+def test_sorted_f_orders_are_permutations_and_batches_sorted():
+    rng = np.random.default_rng(5)
+    for trial in range(40):
+        n = int(rng.integers(1, 13))
+        M = int(rng.integers(12, 90))
+        s, o = random_instance(rng, n, M, M // 2, M // 2)
+        for fn in (lambda: orc.sorted_f_exact(s, o, M, orc.ENUM_ALG1), lambda: orc.sorted_f_exact(s, o, M, orc.ENUM_SUM),
+                   lambda: orc.sorted_f_exact(s, o, M, orc.DP), lambda: orc.sorted_f_prefix(s, o, M)):
+            order, offs = fn()
+            assert sorted(order.tolist()) == list(range(n))
+            assert offs[0] == 0 and offs[-1] == n and (np.diff(offs) > 0).all()
+            for a, b in zip(offs[:-1], offs[1:]):
+                assert (np.diff(o[order[a:b]]) >= 0).all()
+
+
+def test_prefix_f_by_hand():
+    # sizes s+o: r0=4 (o=3), r1=3 (o=1), r2=9 (o=2), r3=5 (o=5); M = 12
+    s = np.array([1, 2, 7, 1], dtype=np.int32)
+    o = np.array([3, 1, 2, 4], dtype=np.int32)
+    # ascending s+o: r1(3), r0(4), r3(5), r2(9); prefixes within M=12: k=1 F=1/1, k=2 F=4/4, k=3 F=8/9 -> k=3
+    order, offs = orc.sorted_f_prefix(s, o, 12)
+    assert offs.tolist() == [0, 3, 4]
+    assert order.tolist() == [1, 0, 3, 2]                  # batch sorted by o: 1, 3, 4
+    # tie on F between k=1 (1/1) and k=2 (4/4) goes to the larger prefix when k=3 does not fit
+    order, offs = orc.sorted_f_prefix(s, o, 9)
+    assert offs.tolist()[:2] == [0, 2]
+
+
+def test_prefix_f_equals_exact_on_homogeneous_types():
+    """Identical requests within a type (Example 2's setting): the best subset is a prefix."""
+    s = np.array([1] * 9 + [30] * 2, dtype=np.int32)
+    o = np.array([2] * 9 + [4] * 2, dtype=np.int32)
+    M = 40
+    o1, f1 = orc.sorted_f_exact(s, o, M, orc.DP)
+    o2, f2 = orc.sorted_f_prefix(s, o, M)
+    assert f1.tolist() == f2.tolist()
+    assert orc.list_schedule_alg1(s, o, M, o1)[1] == orc.list_schedule_alg1(s, o, M, o2)[1]
+
+
+# ----------------------------------------------------------------------------- optimum and the 48x bound
+def test_bruteforce_and_approximation_bound(golden):
+    rng = np.random.default_rng(2024)
+    for trial in range(25):
+        n = int(rng.integers(2, 7))
+        M = int(rng.integers(10, 40))
+        s, o = random_instance(rng, n, M, M // 2, 6)
+        best_list, best_order = orc.bruteforce_best_order(s, o, M)
+        opt, p = orc.bruteforce_opt(s, o, M, best_list + 1)
+        assert 0 < opt <= best_list                        # list schedules are feasible schedules
+        assert orc.check_schedule(s, o, M, p)["feasible"] and orc.check_schedule(s, o, M, p)["tel"] == opt
+        assert opt >= int(o.sum())                         # nobody finishes before decoding o_i tokens
+        for solver in (orc.ENUM_ALG1, orc.ENUM_SUM, orc.DP):
+            order, _ = orc.sorted_f_exact(s, o, M, solver)
+            tel = orc.list_schedule_alg1(s, o, M, order)[1]
+            assert best_list <= tel < golden["approx_ratio_bound"] * opt
+        order, _ = orc.sorted_f_prefix(s, o, M)
+        assert orc.list_schedule_alg1(s, o, M, order)[1] >= best_list
+
+
+def test_bruteforce_on_first_eight_of_tiny_backlog():
+    inst = W.tiny()
+    s, o = inst.s[:8], inst.o[:8]
+    best_list, _ = orc.bruteforce_best_order(s, o, inst.M)
+    opt, p = orc.bruteforce_opt(s, o, inst.M, best_list + 1)
+    assert opt <= best_list and orc.check_schedule(s, o, inst.M, p)["feasible"]
+    order, _ = orc.sorted_f_exact(s, o, inst.M, orc.DP)
+    assert best_list <= orc.list_schedule_alg1(s, o, inst.M, order)[1] < 48 * opt
+
+
+# ----------------------------------------------------------------------------- moves and local search
+def test_move_codes_enumerate_the_neighbourhood():
+    for n in (2, 3, 7, 16):
+        nsw = n * (n - 1) // 2
+        swaps = [orc.decode_move(n, c) for c in range(nsw)]
+        assert [(i, j) for _, i, j in swaps] == list(itertools.combinations(range(n), 2))
+        assert all(t == 0 for t, _, _ in swaps)
+        ins = [orc.decode_move(n, c) for c in range(nsw, nsw + n * (n - 1))]
+        assert [(i, j) for _, i, j in ins] == [(i, j) for i in range(n) for j in range(n) if i != j]
+        assert all(t == 1 for t, _, _ in ins)
+        with pytest.raises(ValueError):
+            orc.decode_move(n, nsw + n * (n - 1))
+        base = np.arange(n, dtype=np.int32)[::-1].copy()
+        for t, i, j in swaps + ins:
+            ref = base.tolist()
+            if t == 0:
+                ref[i], ref[j] = ref[j], ref[i]
+            else:
+                x = ref.pop(i)
+                ref.insert(j, x)
+            assert orc.apply_move(base, t, i, j).tolist() == ref
+            if t == 1:
+                assert ref[j] == base[i]                   # the moved request lands at position j
+
+
+def test_sampled_moves_are_valid_and_reproducible():
+    n = 50
+    seen = set()
+    for m in range(2000):
+        t, i, j = orc.sample_move(n, 42, 3, m)
+        assert t in (0, 1) and 0 <= i < n and 0 <= j < n and i != j
+        if t == 0:
+            assert i < j
+        assert (t, i, j) == orc.sample_move(n, 42, 3, m)
+        seen.add((t, i, j))
+    assert len(seen) > 1500                                # spread over the neighbourhood
+    assert orc.sample_move(n, 42, 4, 0) != orc.sample_move(n, 42, 3, 0) or orc.sample_move(n, 42, 4, 1) != orc.sample_move(n, 42, 3, 1)
+
+
+def test_local_search_descends_to_a_local_optimum():
+    rng = np.random.default_rng(31)
+    for trial in range(8):
+        n = int(rng.integers(4, 9))
+        M = int(rng.integers(14, 40))
+        s, o = random_instance(rng, n, M, M // 2, 6)
+        start = rng.permutation(n).astype(np.int32)
+        t0 = orc.list_schedule_alg1(s, o, M, start)[1]
+        for nb in (orc.SWAP, orc.SWAP_INSERT):
+            order, tel, done, trace = orc.local_search(s, o, M, nb, 100, start)
+            assert sorted(order.tolist()) == list(range(n))
+            assert tel == orc.list_schedule_alg1(s, o, M, order)[1] <= t0
+            accepted = [int(t) for _, t in trace[:-1]]
+            assert accepted == sorted(accepted, reverse=True) and len(set(accepted)) == len(accepted)
+            assert all(t < t0 for t in accepted)
+            # every neighbour of the result is no better (recomputed with the literal executor)
+            ncodes = n * (n - 1) // 2 + (n * (n - 1) if nb == orc.SWAP_INSERT else 0)
+            for c in range(ncodes):
+                cand = orc.apply_move(order, *orc.decode_move(n, c))
+                assert orc.list_schedule_alg1(s, o, M, cand)[1] >= tel
+            assert tel >= orc.bruteforce_best_order(s, o, M)[0]
+
+
+def test_local_search_picks_lowest_code_among_equal_best():
+    # all requests identical: every neighbour ties with the start, nothing is accepted
+    s, o = np.full(6, 3, dtype=np.int32), np.full(6, 2, dtype=np.int32)
+    order, tel, done, trace = orc.local_search(s, o, 11, orc.SWAP_INSERT, 10, np.arange(6))
+    assert done == 1 and trace[0][0] == 0 and order.tolist() == list(range(6))
+
+
+# ----------------------------------------------------------------------------- workloads
+def test_workloads_are_deterministic_and_shaped():
+    a, b = W.mixed_1k(), W.mixed_1k()
+    assert (a.s == b.s).all() and (a.o == b.o).all() and a.checksum() == b.checksum()
+    assert a.checksum() != W.mixed_1k(seed=11).checksum()
+    big = W.mixed_10k()
+    assert big.n == 10000 and big.M == 262144
+    docs = big.s >= 4096
+    assert 0.17 < docs.mean() < 0.23
+    assert big.s[~docs].max() <= 2048 and big.s[~docs].min() >= 16
+    assert big.o[~docs].max() <= 1024 and big.o[~docs].min() >= 8
+    assert big.o[docs].min() >= 128 and big.o[docs].max() <= 512
+    assert (big.s.astype(np.int64) + big.o).sum() > 20 * big.M          # overloaded regime
+    t = W.tiny()
+    assert t.n == 16 and t.s.min() >= 1 and t.s.max() <= 32 and t.o.min() >= 1 and t.o.max() <= 32
