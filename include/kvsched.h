@@ -1,0 +1,171 @@
+/* kvsched -- batched evaluation of KV-cache-constrained request schedules on one GPU (sm_100a).
+ *
+ * Problem (paper, Section 2.1-2.2): n requests, all present at t = 0; request i has a prefill
+ * length s_i and a decode length o_i; a single worker holds at most M tokens of KV cache.  A request
+ * that starts at p_i >= 0 is resident in rounds p_i+1 .. p_i+o_i, uses s_i + (tau - p_i) tokens in
+ * round tau, and completes at c_i = p_i + o_i (integer program of Section 6.1).  A schedule is
+ * feasible iff the total usage never exceeds M; its cost is the total end-to-end latency
+ * TEL = sum_i c_i, in rounds.
+ *
+ * An ORDER (a permutation of the requests) is turned into start times by Phase 2 of Algorithm 1
+ * (Appendix C): every round, finished requests leave, then pending requests are admitted in list
+ * order for as long as the memory of all running requests stays within M at every future round;
+ * the first request that does not fit ends that round's admissions.
+ *
+ * Conventions of this interface
+ *   - Every function returns SCHED_OK (0) or a negative SCHED_E_* code; nothing throws, and no GPU
+ *     trap is ever used to report an error.  sched_strerror() names a code.
+ *   - "host" pointers are ordinary CPU memory; "device" pointers are memory of the handle's GPU.
+ *     The plain entry points take host pointers, copy in/out, and return when results are in the
+ *     caller's buffers.  The *_dev entry points take device pointers, enqueue on the handle's
+ *     stream and return without synchronising (sched_sync() waits).
+ *   - The caller owns every buffer it passes.  The handle owns device copies of (s, o), the base
+ *     order and all scratch memory; sched_destroy() frees them.
+ *   - A handle is tied to the CUDA device that was current in sched_init(); calls on one handle
+ *     must not overlap in time.
+ *   - Arrays are dense, row-major, int32 unless stated; TELs are int64.
+ */
+#ifndef KVSCHED_H
+#define KVSCHED_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct sched_ctx* sched_handle;
+
+enum {
+    SCHED_OK = 0,
+    SCHED_E_INVAL = -1,            /* bad argument: n <= 0, s_i < 1, o_i < 1, M < 1, s_i + o_i > M, ... */
+    SCHED_E_NOT_PERMUTATION = -2,  /* an ORDER candidate (or order_inout) is not a permutation of 0..n-1 */
+    SCHED_E_CUDA = -3,             /* a CUDA runtime call failed (sched_last_cuda_error() has the text) */
+    SCHED_E_NOMEM = -4,            /* host or device allocation failed */
+    SCHED_E_INTERNAL = -5,         /* a bounded device loop hit its cap; results are not valid */
+    SCHED_E_UNSUPPORTED = -6       /* sizes beyond what this build handles (see each call) */
+};
+
+/* What one candidate of sched_eval_batch() is. */
+enum {
+    SCHED_CAND_ORDER = 0,        /* int32[count][n]: a permutation; list-scheduled, always feasible     */
+    SCHED_CAND_MOVE = 1,         /* int64[count]: move codes relative to the handle's base order         */
+    SCHED_CAND_START_TIMES = 2,  /* int32[count][n]: explicit starts p_i; checked against the budget     */
+    SCHED_CAND_POLICY = 3        /* int32[count]: SCHED_POLICY_* ids; each instance x each policy        */
+};
+
+/* Order policies (Section 2.3, Appendix A, Section 7). Ties always go to the lower request index. */
+enum {
+    SCHED_POLICY_FCFS = 0,        /* index order                                                         */
+    SCHED_POLICY_SOF = 1,         /* shortest output first (MC-SF): ascending o                          */
+    SCHED_POLICY_TOTAL_SIZE = 2,  /* smallest s+o first (MC-SF_2)                                        */
+    SCHED_POLICY_SORTED_F = 3     /* Sorted-F with prefix-F batch selection, see sched_sorted_f()        */
+};
+
+/* Local-search neighbourhoods over positions of the base order.
+ * Move codes: swap(i,j), 0 <= i < j < n, in lexicographic order, codes 0 .. n(n-1)/2 - 1; then
+ * insert(i -> j), i != j (take the request at position i out and put it back so that it sits at
+ * position j), code n(n-1)/2 + i*(n-1) + (j < i ? j : j-1). */
+enum {
+    SCHED_NBHD_SWAP = 0,         /* all n(n-1)/2 swaps                                                   */
+    SCHED_NBHD_SWAP_INSERT = 1,  /* all swaps, then all n(n-1) inserts                                   */
+    SCHED_NBHD_SAMPLED = 2       /* samples_per_iter moves per iteration from a counter-based hash       */
+};
+
+/* Create a handle for one instance (paper, Section 2.1: n, (s_i, o_i), M).
+ *   s, o : host int32[n], copied.  Requires n >= 1, s_i >= 1, o_i >= 1, M >= 1 and s_i + o_i <= M
+ *          (the paper's standing assumption; otherwise Algorithm 1 would never admit the request),
+ *          else SCHED_E_INVAL.  SCHED_E_UNSUPPORTED if sum(o_i) + max(o_i) >= 2^30 or M >= 2^30.
+ *   The base order starts as the identity. */
+int sched_init(sched_handle* out, int32_t n, const int32_t* s, const int32_t* o, int64_t M);
+
+/* Create a handle for B independent instances of n_each requests each (policy sweeps).
+ *   s, o : host int32[B][n_each].  Same checks as sched_init for every instance.
+ *   Only sched_eval_batch(SCHED_CAND_POLICY) is available on such a handle. n_each <= 1024. */
+int sched_init_batch(sched_handle* out, int32_t B, int32_t n_each, const int32_t* s, const int32_t* o, int64_t M);
+
+/* Use an existing CUDA stream (a cudaStream_t passed as void*) for all work of this handle.
+ * NULL selects the handle's own stream again. */
+int sched_set_stream(sched_handle h, void* cuda_stream);
+
+/* Wait for everything enqueued on the handle's stream; reports device-side status
+ * (SCHED_E_INTERNAL if any bounded loop gave up since the last call). */
+int sched_sync(sched_handle h);
+
+/* Base order used by SCHED_CAND_MOVE candidates and by sched_local_search(). host int32[n]. */
+int sched_set_base_order(sched_handle h, const int32_t* order);
+int sched_get_base_order(sched_handle h, int32_t* order_out);
+
+/* Evaluate `count` candidates at once (Algorithm 1 Phase 2 for ORDER / MOVE / POLICY; the memory
+ * row and objective of the integer program, Section 6.1, for START_TIMES).
+ *   candidates   : layout per `kind`, see SCHED_CAND_*.
+ *   tel_out      : int64[count] (POLICY: int64[B][count]).  START_TIMES: sum(p_i + o_i), also when
+ *                  infeasible.
+ *   feasible_out : uint8[count], nullable.  1 unless a START_TIMES candidate exceeds M in some round
+ *                  (ORDER / MOVE / POLICY candidates are feasible by construction).
+ *   starts_out   : nullable; int32[count][n] start time p_i of every request i, indexed by request
+ *                  id (ORDER, MOVE, and POLICY with layout [B][count][n_each]).
+ * Host-pointer form: validates ORDER candidates (SCHED_E_NOT_PERMUTATION), MOVE codes and policy
+ * ids (SCHED_E_INVAL) and negative start times (SCHED_E_INVAL) before any launch. */
+int sched_eval_batch(sched_handle h, int kind, int64_t count, const void* candidates,
+                     int64_t* tel_out, uint8_t* feasible_out, int32_t* starts_out);
+
+/* Same, device pointers, asynchronous on the handle's stream, candidates not validated. */
+int sched_eval_batch_dev(sched_handle h, int kind, int64_t count, const void* candidates,
+                         int64_t* tel_out, uint8_t* feasible_out, int32_t* starts_out);
+
+/* Evaluate the contiguous move-code range [first_code, first_code + count) (SWAP_INSERT coding)
+ * against the base order, or -- if sampled != 0 -- the sampled moves m = first_code .. first_code +
+ * count - 1 of iteration `iteration` under `seed`; then reduce to the best (TEL, index) pair.
+ *   tel_out  : device int64[count], nullable (per-candidate TELs are still reduced if NULL).
+ *   best_out : device int64[2] = {min TEL, lowest index (code or m) attaining it}.
+ * Asynchronous on the handle's stream.  This is one neighbourhood sweep of sched_local_search(). */
+int sched_sweep_dev(sched_handle h, int sampled, uint64_t seed, int32_t iteration,
+                    int64_t first_code, int64_t count, int64_t* tel_out, int64_t* best_out);
+
+/* Sorted-F (Algorithm 1 Phase 1 + Phase 2) with prefix-F batch selection: requests are sorted by
+ * (s+o, o, index) ascending -- the order Algorithm 4 starts from; from the current offset a, with
+ * k_max the longest prefix of the remaining requests whose sum(s+o) <= M, the batch is the prefix
+ * of length k* = argmin_{1<=k<=k_max} (sum of o over the prefix) / k^2, ties to the larger k
+ * (Section 3: minimise F, prefer the larger batch; compared exactly in integers); the batch is
+ * sorted by (o, index) and appended.  The resulting order becomes the handle's base order.
+ *   order_out         : host int32[n], nullable.
+ *   batch_offsets_out : host int32[n+1], nullable; entries 0..num_batches are filled.
+ *   num_batches_out, tel_out : nullable. */
+int sched_sorted_f(sched_handle h, int32_t* order_out, int32_t* batch_offsets_out,
+                   int32_t* num_batches_out, int64_t* tel_out);
+
+/* Same, results left on the device; asynchronous.  order_out int32[n], batch_offsets_out
+ * int32[n+1], num_batches_out int32[1], tel_out int64[1]; each nullable. */
+int sched_sorted_f_dev(sched_handle h, int32_t* order_out, int32_t* batch_offsets_out,
+                       int32_t* num_batches_out, int64_t* tel_out);
+
+/* Order-level local search from order_inout (NULL: from the handle's base order).  Each iteration
+ * evaluates the whole neighbourhood with Algorithm 1 Phase 2, takes the best (TEL, code) pair --
+ * lowest code among equal TELs -- and accepts it iff its TEL is strictly below the current one
+ * (Section 5.2's improving-swap rule applied to list positions).  SWAP / SWAP_INSERT stop at the
+ * first iteration without an improving move (that iteration is counted); SAMPLED always runs
+ * `iters` iterations, drawing move m of iteration it from h1 = mix(seed ^ mix(it * 2^32 + m)),
+ * h2 = mix(h1) (mix = splitmix64 step): type = h1 & 1, i = (h1 >> 1) mod n,
+ * j = (i + 1 + h2 mod (n-1)) mod n, a swap normalised to i < j.
+ *   order_inout    : host int32[n], nullable; receives the final order.
+ *   tel_out        : final TEL.  iters_done_out: iterations executed.  Both nullable.
+ *   trace_out      : nullable host int64[iters][2]: per iteration {best code, best TEL}.
+ * The final order becomes the handle's base order, so a run can be resumed by calling again. */
+int sched_local_search(sched_handle h, int neighbourhood, int32_t iters, uint64_t seed,
+                       int64_t samples_per_iter, int32_t* order_inout, int64_t* tel_out,
+                       int32_t* iters_done_out, int64_t* trace_out);
+
+/* Counters since sched_init: kernels launched by this handle, candidates evaluated. */
+int sched_stats(sched_handle h, int64_t* kernel_launches_out, int64_t* evaluations_out);
+
+int sched_destroy(sched_handle h);
+
+const char* sched_strerror(int code);
+/* Text of the last CUDA error seen by this library on the calling thread ("" if none). */
+const char* sched_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KVSCHED_H */

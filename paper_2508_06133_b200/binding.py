@@ -1,0 +1,222 @@
+"""Thin ctypes binding of the kvsched C-ABI (``include/kvsched.h``): argument marshalling only.
+
+Every step of the path runs in the CUDA library; this module allocates nothing but numpy / torch
+buffers for inputs and outputs and raises ``SchedError`` on any non-zero return code.  There is no
+CPU fallback: if ``libkvsched.so`` is missing, importing the library fails with instructions.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libkvsched.so")
+
+OK, E_INVAL, E_NOT_PERMUTATION, E_CUDA, E_NOMEM, E_INTERNAL, E_UNSUPPORTED = 0, -1, -2, -3, -4, -5, -6
+CAND_ORDER, CAND_MOVE, CAND_START_TIMES, CAND_POLICY = 0, 1, 2, 3
+POLICY_FCFS, POLICY_SOF, POLICY_TOTAL_SIZE, POLICY_SORTED_F = 0, 1, 2, 3
+NBHD_SWAP, NBHD_SWAP_INSERT, NBHD_SAMPLED = 0, 1, 2
+
+EXPORTS = [
+    "sched_init", "sched_init_batch", "sched_set_stream", "sched_sync", "sched_set_base_order",
+    "sched_get_base_order", "sched_eval_batch", "sched_eval_batch_dev", "sched_sweep_dev",
+    "sched_sorted_f", "sched_sorted_f_dev", "sched_local_search", "sched_stats", "sched_destroy",
+    "sched_strerror", "sched_last_cuda_error",
+]
+
+_lib = None
+
+
+class SchedError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        l = load()
+        msg = l.sched_strerror(code).decode()
+        cuda = l.sched_last_cuda_error().decode()
+        super().__init__("%s failed: %s (%d)%s" % (where, msg, code, (" [" + cuda + "]") if cuda and code == E_CUDA else ""))
+
+
+def load():
+    """Load libkvsched.so (after torch, so that both share one CUDA runtime)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError("libkvsched.so is not built: run `python -m paper_2508_06133_b200.build` "
+                          "(needs nvcc; there is no CPU fallback)")
+    try:
+        import torch  # noqa: F401  (loads libcudart)
+    except Exception:  # pragma: no cover
+        pass
+    lib = C.CDLL(LIB_PATH)
+    vp, i32, i64, u64 = C.c_void_p, C.c_int32, C.c_int64, C.c_uint64
+    lib.sched_init.argtypes = [C.POINTER(vp), i32, vp, vp, i64]
+    lib.sched_init_batch.argtypes = [C.POINTER(vp), i32, i32, vp, vp, i64]
+    lib.sched_set_stream.argtypes = [vp, vp]
+    lib.sched_sync.argtypes = [vp]
+    lib.sched_set_base_order.argtypes = [vp, vp]
+    lib.sched_get_base_order.argtypes = [vp, vp]
+    lib.sched_eval_batch.argtypes = [vp, C.c_int, i64, vp, vp, vp, vp]
+    lib.sched_eval_batch_dev.argtypes = [vp, C.c_int, i64, vp, vp, vp, vp]
+    lib.sched_sweep_dev.argtypes = [vp, C.c_int, u64, i32, i64, i64, vp, vp]
+    lib.sched_sorted_f.argtypes = [vp, vp, vp, vp, vp]
+    lib.sched_sorted_f_dev.argtypes = [vp, vp, vp, vp, vp]
+    lib.sched_local_search.argtypes = [vp, C.c_int, i32, u64, i64, vp, vp, vp, vp]
+    lib.sched_stats.argtypes = [vp, vp, vp]
+    lib.sched_destroy.argtypes = [vp]
+    lib.sched_strerror.argtypes = [C.c_int]
+    lib.sched_strerror.restype = C.c_char_p
+    lib.sched_last_cuda_error.argtypes = []
+    lib.sched_last_cuda_error.restype = C.c_char_p
+    for name in EXPORTS:
+        if name not in ("sched_strerror", "sched_last_cuda_error"):
+            getattr(lib, name).restype = C.c_int
+    _lib = lib
+    return lib
+
+
+def _np_ptr(a):
+    return a.ctypes.data_as(C.c_void_p) if a is not None else None
+
+
+def _dev_ptr(t):
+    """Device pointer of a contiguous CUDA torch tensor (or None)."""
+    if t is None:
+        return None
+    assert t.is_cuda and t.is_contiguous()
+    return C.c_void_p(t.data_ptr())
+
+
+def _check(rc, where):
+    if rc != OK:
+        raise SchedError(rc, where)
+
+
+class Scheduler:
+    """One handle of the C library.  Methods mirror the C entry points one to one."""
+
+    def __init__(self, s, o, M, *, batch=None):
+        lib = load()
+        s = np.ascontiguousarray(s, dtype=np.int32)
+        o = np.ascontiguousarray(o, dtype=np.int32)
+        self._h = C.c_void_p()
+        self.M = int(M)
+        if batch is None:
+            self.B, self.n = 1, int(s.shape[0])
+            rc = lib.sched_init(C.byref(self._h), self.n, _np_ptr(s), _np_ptr(o), self.M)
+            where = "sched_init"
+        else:
+            self.B, self.n = int(s.shape[0]), int(s.shape[1])
+            rc = lib.sched_init_batch(C.byref(self._h), self.B, self.n, _np_ptr(s), _np_ptr(o), self.M)
+            where = "sched_init_batch"
+        if rc != OK:
+            self._h = None
+            raise SchedError(rc, where)
+
+    @classmethod
+    def batch(cls, s, o, M):
+        return cls(s, o, M, batch=True)
+
+    # ---- lifetime
+    def close(self):
+        if getattr(self, "_h", None):
+            load().sched_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.close()
+
+    # ---- plumbing
+    def set_stream(self, stream=None):
+        """``stream``: a torch.cuda.Stream (or None for the handle's own stream)."""
+        ptr = C.c_void_p(stream.cuda_stream) if stream is not None else None
+        _check(load().sched_set_stream(self._h, ptr), "sched_set_stream")
+
+    def sync(self):
+        _check(load().sched_sync(self._h), "sched_sync")
+
+    def stats(self):
+        a, b = C.c_int64(0), C.c_int64(0)
+        _check(load().sched_stats(self._h, C.byref(a), C.byref(b)), "sched_stats")
+        return a.value, b.value
+
+    def set_base_order(self, order):
+        order = np.ascontiguousarray(order, dtype=np.int32)
+        if order.shape != (self.n,):
+            raise SchedError(E_INVAL, "sched_set_base_order")
+        _check(load().sched_set_base_order(self._h, _np_ptr(order)), "sched_set_base_order")
+
+    def get_base_order(self):
+        out = np.empty(self.n, dtype=np.int32)
+        _check(load().sched_get_base_order(self._h, _np_ptr(out)), "sched_get_base_order")
+        return out
+
+    # ---- sched_eval_batch (host buffers)
+    def eval_batch(self, kind, candidates, *, want_feasible=False, want_starts=False):
+        """Returns (tel, feasible or None, starts or None) as numpy arrays."""
+        if kind in (CAND_ORDER, CAND_START_TIMES):
+            cand = np.ascontiguousarray(candidates, dtype=np.int32).reshape(-1, self.n)
+            count, outs = cand.shape[0], cand.shape[0]
+        elif kind == CAND_MOVE:
+            cand = np.ascontiguousarray(candidates, dtype=np.int64).reshape(-1)
+            count, outs = cand.shape[0], cand.shape[0]
+        else:
+            cand = np.ascontiguousarray(candidates, dtype=np.int32).reshape(-1)
+            count, outs = cand.shape[0], cand.shape[0] * self.B
+        tel = np.empty(outs, dtype=np.int64)
+        feas = np.empty(outs, dtype=np.uint8) if want_feasible else None
+        starts = np.empty((outs, self.n), dtype=np.int32) if want_starts else None
+        _check(load().sched_eval_batch(self._h, kind, count, _np_ptr(cand), _np_ptr(tel), _np_ptr(feas), _np_ptr(starts)),
+               "sched_eval_batch")
+        if kind == CAND_POLICY:
+            tel = tel.reshape(self.B, count)
+            feas = feas.reshape(self.B, count) if feas is not None else None
+            starts = starts.reshape(self.B, count, self.n) if starts is not None else None
+        return tel, feas, starts
+
+    # ---- device-pointer forms (torch CUDA tensors); asynchronous
+    def eval_batch_dev(self, kind, count, candidates, tel_out, feasible_out=None, starts_out=None):
+        _check(load().sched_eval_batch_dev(self._h, kind, count, _dev_ptr(candidates), _dev_ptr(tel_out),
+                                           _dev_ptr(feasible_out), _dev_ptr(starts_out)), "sched_eval_batch_dev")
+
+    def sweep_dev(self, count, best_out, *, first_code=0, sampled=False, seed=0, iteration=0, tel_out=None):
+        _check(load().sched_sweep_dev(self._h, 1 if sampled else 0, seed, iteration, first_code, count,
+                                      _dev_ptr(tel_out), _dev_ptr(best_out)), "sched_sweep_dev")
+
+    def sorted_f_dev(self, order_out=None, batch_offsets_out=None, num_batches_out=None, tel_out=None):
+        _check(load().sched_sorted_f_dev(self._h, _dev_ptr(order_out), _dev_ptr(batch_offsets_out),
+                                         _dev_ptr(num_batches_out), _dev_ptr(tel_out)), "sched_sorted_f_dev")
+
+    # ---- sched_sorted_f / sched_local_search (host buffers)
+    def sorted_f(self):
+        """Returns (order, batch_offsets[0..num_batches], TEL)."""
+        order = np.empty(self.n, dtype=np.int32)
+        offs = np.zeros(self.n + 1, dtype=np.int32)
+        nb, tel = C.c_int32(0), C.c_int64(0)
+        _check(load().sched_sorted_f(self._h, _np_ptr(order), _np_ptr(offs), C.byref(nb), C.byref(tel)), "sched_sorted_f")
+        return order, offs[:nb.value + 1].copy(), tel.value
+
+    def local_search(self, neighbourhood, iters, *, order=None, seed=0, samples_per_iter=0):
+        """Returns (final order, TEL, iterations done, trace[(code, best TEL)])."""
+        buf = None
+        if order is not None:
+            buf = np.ascontiguousarray(order, dtype=np.int32).copy()
+            if buf.shape != (self.n,):
+                raise SchedError(E_INVAL, "sched_local_search")
+        trace = np.full((max(iters, 1), 2), -1, dtype=np.int64)
+        tel, done = C.c_int64(0), C.c_int32(0)
+        _check(load().sched_local_search(self._h, neighbourhood, iters, seed, samples_per_iter, _np_ptr(buf),
+                                         C.byref(tel), C.byref(done), _np_ptr(trace)), "sched_local_search")
+        final = buf if buf is not None else self.get_base_order()
+        return final, tel.value, done.value, trace[:done.value].copy()

@@ -1,0 +1,606 @@
+// Host side of the kvsched C-ABI (see include/kvsched.h for the contract of every entry point).
+// All scheduling arithmetic runs in the kernels of k1_sort / k2_fmetric / k3_eval / k5_argmin; this
+// file validates arguments, owns device memory and enqueues launches.  There is no CPU fallback.
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "common.cuh"
+#include "k1_sort.cuh"
+#include "k2_fmetric.cuh"
+#include "k3_eval.cuh"
+#include "k5_argmin.cuh"
+
+thread_local char g_last_cuda_error[256] = "";
+
+int kv_cuda_fail(cudaError_t e, const char* what) {
+    snprintf(g_last_cuda_error, sizeof(g_last_cuda_error), "%s: %s", what, cudaGetErrorString(e));
+    return e == cudaErrorMemoryAllocation ? SCHED_E_NOMEM : SCHED_E_CUDA;
+}
+
+namespace {
+
+const i64 kSweepChunk = 1ll << 22;          // candidates per launch inside a sweep
+const size_t kSnapBudget = 512ull << 20;    // bytes of snapshot memory before striding kicks in
+
+int bits_of(u64 v) { int b = 0; while (v) { ++b; v >>= 1; } return b; }
+
+// byte mask for a 64-bit key whose low word uses lo_bits and high word hi_bits
+unsigned key_byte_mask(int lo_bits, int hi_bits) {
+    unsigned m = 0;
+    for (int b = 0; b < (lo_bits + 7) / 8; ++b) m |= 1u << b;
+    for (int b = 0; b < (hi_bits + 7) / 8; ++b) m |= 1u << (4 + b);
+    return m;
+}
+
+template <typename T>
+int dev_alloc(T** p, size_t count) {
+    *p = nullptr;
+    if (count == 0) count = 1;
+    KV_CUDA(cudaMalloc((void**)p, count * sizeof(T)));
+    return SCHED_OK;
+}
+
+int ensure_stage(sched_ctx* h, size_t bytes) {
+    if (h->stage_cap >= bytes) return SCHED_OK;
+    if (h->d_stage) { cudaFree(h->d_stage); h->d_stage = nullptr; h->stage_cap = 0; }
+    KV_CUDA(cudaMalloc(&h->d_stage, bytes));
+    h->stage_cap = bytes;
+    return SCHED_OK;
+}
+
+int ensure_tel(sched_ctx* h, i64 count) {
+    if (h->tel_cap >= count) return SCHED_OK;
+    if (h->d_tel) { cudaFree(h->d_tel); h->d_tel = nullptr; h->tel_cap = 0; }
+    KV_TRY(dev_alloc(&h->d_tel, (size_t)count + 2));
+    h->tel_cap = count;
+    return SCHED_OK;
+}
+
+struct DeviceGuard {
+    int prev;
+    bool ok;
+    explicit DeviceGuard(int dev) : prev(-1), ok(false) {
+        if (cudaGetDevice(&prev) != cudaSuccess) return;
+        ok = (prev == dev) || cudaSetDevice(dev) == cudaSuccess;
+    }
+    ~DeviceGuard() { if (ok && prev >= 0) cudaSetDevice(prev); }
+};
+
+#define KV_ENTER(h)                                                  \
+    if (!(h)) return SCHED_E_INVAL;                                  \
+    DeviceGuard guard__((h)->device);                                \
+    if (!guard__.ok) return kv_cuda_fail(cudaGetLastError(), "cudaSetDevice")
+
+int check_launch(sched_ctx* h) {
+    h->launches += 1;
+    KV_CUDA(cudaGetLastError());
+    return SCHED_OK;
+}
+
+int validate_instance(i64 total, const int32_t* s, const int32_t* o, i64 M) {
+    for (i64 i = 0; i < total; ++i) {
+        if (s[i] < 1 || o[i] < 1) return SCHED_E_INVAL;
+        if ((i64)s[i] + (i64)o[i] > M) return SCHED_E_INVAL;
+    }
+    return SCHED_OK;
+}
+
+void free_ctx(sched_ctx* h) {
+    if (!h) return;
+    void* ptrs[] = {h->d_s, h->d_o, h->d_tbl_id, h->d_tbl_base, h->d_order, h->d_snap_ring, h->d_snap_hdr,
+                    h->d_base_tel, h->d_counter, h->d_status, h->d_tel, h->d_best, h->d_partials, h->d_ticket,
+                    h->d_keys_a, h->d_keys_b, h->d_vals_a, h->d_vals_b, h->d_prefP, h->d_prefO,
+                    h->d_batch_off, h->d_num_batches, h->d_seg_off, h->d_stage, h->d_base_starts,
+                    h->d_state, h->d_sort};
+    for (void* p : ptrs) if (p) cudaFree(p);
+    if (h->h_pinned) cudaFreeHost(h->h_pinned);
+    if (h->own_stream) cudaStreamDestroy(h->own_stream);
+    delete h;
+}
+
+size_t k3_smem_bytes(const sched_ctx* h, bool* table_in_smem, unsigned* table_bytes) {
+    const size_t rings = (size_t)K3_WARPS * h->L * sizeof(int);
+    const unsigned tb = (unsigned)(((size_t)h->n * sizeof(int2) + 15) & ~(size_t)15);
+    const size_t with_table = ((size_t)tb + 127) / 128 * 128 + rings;
+    if (with_table <= (size_t)h->smem_optin - 1024) {
+        *table_in_smem = true; *table_bytes = tb; return with_table;
+    }
+    *table_in_smem = false; *table_bytes = tb; return rings;
+}
+
+int create_common(sched_ctx** out, int B, int n, const int32_t* s, const int32_t* o, i64 M) {
+    if (!out) return SCHED_E_INVAL;
+    *out = nullptr;
+    if (B < 1 || n < 1 || !s || !o || M < 1) return SCHED_E_INVAL;
+    if (M >= (1ll << 30)) return SCHED_E_UNSUPPORTED;
+    const i64 total = (i64)B * n;
+    KV_TRY(validate_instance(total, s, o, M));
+    int omax = 0; i64 sum_max = 0;
+    for (int b = 0; b < B; ++b) {
+        i64 sum = 0;
+        for (int i = 0; i < n; ++i) { int v = o[(i64)b * n + i]; sum += v; if (v > omax) omax = v; }
+        if (sum > sum_max) sum_max = sum;
+    }
+    if (sum_max + omax >= (1ll << 30)) return SCHED_E_UNSUPPORTED;
+
+    sched_ctx* h = new (std::nothrow) sched_ctx();
+    if (!h) return SCHED_E_NOMEM;
+    memset(h, 0, sizeof(*h));
+    int rc = SCHED_OK;
+    do {
+        if (cudaGetDevice(&h->device) != cudaSuccess) { rc = kv_cuda_fail(cudaGetLastError(), "cudaGetDevice"); break; }
+        cudaDeviceProp prop;
+        if (cudaGetDeviceProperties(&prop, h->device) != cudaSuccess) { rc = kv_cuda_fail(cudaGetLastError(), "cudaGetDeviceProperties"); break; }
+        h->sm_count = prop.multiProcessorCount;
+        h->smem_optin = (int)prop.sharedMemPerBlockOptin;
+        h->B = B; h->n = n; h->M = M; h->omax = omax; h->sum_o_max = sum_max;
+        h->L = (omax + 8 + 3) & ~3;
+        if ((size_t)K3_WARPS * h->L * sizeof(int) > (size_t)h->smem_optin - 1024) { rc = SCHED_E_UNSUPPORTED; break; }
+        if (cudaStreamCreateWithFlags(&h->own_stream, cudaStreamNonBlocking) != cudaSuccess) { rc = kv_cuda_fail(cudaGetLastError(), "cudaStreamCreate"); break; }
+        h->stream = h->own_stream;
+#define A(call) if ((rc = (call)) != SCHED_OK) break
+        A(dev_alloc(&h->d_s, total)); A(dev_alloc(&h->d_o, total));
+        A(dev_alloc(&h->d_tbl_id, total + 2));
+        A(dev_alloc(&h->d_counter, 4)); A(dev_alloc(&h->d_status, 1));
+        A(dev_alloc(&h->d_best, 2)); A(dev_alloc(&h->d_partials, 2 * 4096)); A(dev_alloc(&h->d_ticket, 1));
+        A(dev_alloc(&h->d_state, 4));
+        if (cudaMallocHost(&h->h_pinned, 64) != cudaSuccess) { rc = kv_cuda_fail(cudaGetLastError(), "cudaMallocHost"); break; }
+        if (B == 1) {
+            A(dev_alloc(&h->d_tbl_base, n + 2)); A(dev_alloc(&h->d_order, n));
+            A(dev_alloc(&h->d_base_starts, n)); A(dev_alloc(&h->d_base_tel, 1));
+            A(dev_alloc(&h->d_keys_a, n)); A(dev_alloc(&h->d_keys_b, n));
+            A(dev_alloc(&h->d_vals_a, n)); A(dev_alloc(&h->d_vals_b, n));
+            A(dev_alloc(&h->d_prefP, n + 1)); A(dev_alloc(&h->d_prefO, n + 1));
+            A(dev_alloc(&h->d_batch_off, n + 1)); A(dev_alloc(&h->d_num_batches, 1)); A(dev_alloc(&h->d_seg_off, 2));
+            size_t per = (size_t)h->L * sizeof(int);
+            i64 stride = (i64)(((size_t)n * per + kSnapBudget - 1) / kSnapBudget);
+            if (stride < 1) stride = 1;
+            h->snap_stride = (int)stride;
+            h->snap_count = (n + h->snap_stride - 1) / h->snap_stride;
+            A(dev_alloc(&h->d_snap_ring, (size_t)h->snap_count * h->L));
+            A(dev_alloc(&h->d_snap_hdr, h->snap_count));
+        }
+#undef A
+        cudaStream_t st = h->stream;
+#define C(call) if ((call) != cudaSuccess) { rc = kv_cuda_fail(cudaGetLastError(), #call); break; }
+        C(cudaMemcpyAsync(h->d_s, s, total * sizeof(int), cudaMemcpyHostToDevice, st));
+        C(cudaMemcpyAsync(h->d_o, o, total * sizeof(int), cudaMemcpyHostToDevice, st));
+        C(cudaMemsetAsync(h->d_tbl_id, 0, (total + 2) * sizeof(int2), st));
+        C(cudaMemsetAsync(h->d_status, 0, sizeof(int), st));
+        C(cudaMemsetAsync(h->d_ticket, 0, sizeof(unsigned), st));
+        C(cudaMemsetAsync(h->d_counter, 0, 4 * sizeof(unsigned), st));
+        k3_make_table<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(h->d_s, h->d_o, (int)total, h->d_tbl_id);
+        if ((rc = check_launch(h)) != SCHED_OK) break;
+        if (B == 1) {
+            C(cudaMemsetAsync(h->d_tbl_base, 0, (n + 2) * sizeof(int2), st));
+            k3_iota<<<(n + 255) / 256, 256, 0, st>>>(h->d_order, n);
+            if ((rc = check_launch(h)) != SCHED_OK) break;
+            int seg[2] = {0, n};
+            C(cudaMemcpyAsync(h->d_seg_off, seg, sizeof(seg), cudaMemcpyHostToDevice, st));
+        }
+        // opt in to large dynamic shared memory once
+        C(cudaFuncSetAttribute(k3_eval_moves, cudaFuncAttributeMaxDynamicSharedMemorySize, h->smem_optin - 1024));
+        C(cudaFuncSetAttribute(k3_eval_orders, cudaFuncAttributeMaxDynamicSharedMemorySize, h->smem_optin - 1024));
+        C(cudaFuncSetAttribute(k3_check_starts, cudaFuncAttributeMaxDynamicSharedMemorySize, h->smem_optin - 1024));
+        C(cudaFuncSetAttribute(k3_eval_policy, cudaFuncAttributeMaxDynamicSharedMemorySize, h->smem_optin - 1024));
+        C(cudaFuncSetAttribute(k3_base_run, cudaFuncAttributeMaxDynamicSharedMemorySize, h->smem_optin - 1024));
+        C(cudaStreamSynchronize(st));       // s, o may be pageable host memory owned by the caller
+#undef C
+    } while (0);
+    if (rc != SCHED_OK) { free_ctx(h); return rc; }
+    *out = h;
+    return SCHED_OK;
+}
+
+// Base order -> position-ordered table, snapshots, base TEL.
+int ensure_base(sched_ctx* h) {
+    if (h->base_ready) return SCHED_OK;
+    const int n = h->n;
+    k3_gather_table<<<(n + 255) / 256, 256, 0, h->stream>>>(h->d_tbl_id, h->d_order, n, h->d_tbl_base);
+    KV_TRY(check_launch(h));
+    k3_base_run<<<1, 32, (size_t)h->L * sizeof(int), h->stream>>>(
+        h->d_tbl_base, n, h->L, (int)h->M, h->snap_stride, h->d_snap_ring, h->d_snap_hdr,
+        h->d_base_starts, h->d_base_tel, h->d_status);
+    KV_TRY(check_launch(h));
+    h->base_ready = true;
+    return SCHED_OK;
+}
+
+int k3_grid(const sched_ctx* h, i64 count) {
+    i64 ctas = (count + K3_WARPS - 1) / K3_WARPS;
+    if (ctas > h->sm_count) ctas = h->sm_count;
+    if (ctas < 1) ctas = 1;
+    return (int)ctas;
+}
+
+int launch_moves(sched_ctx* h, int mode, const i64* codes, i64 first, u64 seed, int iteration,
+                 i64 count, i64* tel_out, int* starts_out) {
+    if (count <= 0) return SCHED_OK;
+    if (count >= (1ll << 31)) return SCHED_E_UNSUPPORTED;
+    KV_TRY(ensure_base(h));
+    MoveEvalParams p;
+    memset(&p, 0, sizeof(p));
+    bool in_smem; unsigned tb;
+    const size_t smem = k3_smem_bytes(h, &in_smem, &tb);
+    p.n = h->n; p.L = h->L; p.M = (int)h->M; p.stride = h->snap_stride;
+    p.tbl_base = h->d_tbl_base; p.table_in_smem = in_smem ? 1 : 0; p.table_bytes = tb;
+    p.snap_ring = h->d_snap_ring; p.snap_hdr = h->d_snap_hdr;
+    p.mode = mode; p.codes = codes; p.first = first; p.seed = seed; p.iteration = iteration;
+    p.count = count; p.tel_out = tel_out; p.starts_out = starts_out;
+    p.base_order = h->d_order; p.base_starts_pos = h->d_base_starts;
+    p.counter = h->d_counter; p.status = h->d_status;
+    KV_CUDA(cudaMemsetAsync(h->d_counter, 0, sizeof(unsigned), h->stream));
+    k3_eval_moves<<<k3_grid(h, count), K3_THREADS, smem, h->stream>>>(p);
+    KV_TRY(check_launch(h));
+    h->evaluations += count;
+    return SCHED_OK;
+}
+
+int launch_argmin(sched_ctx* h, const i64* tel, i64 count, i64 index_base, const i64* prior, i64* best_out) {
+    i64 blocks = (count / 2 + K5_THREADS - 1) / K5_THREADS;
+    if (blocks < 1) blocks = 1;
+    if (blocks > 4 * h->sm_count) blocks = 4 * h->sm_count;
+    if (blocks > 4096) blocks = 4096;
+    k5_argmin<<<(unsigned)blocks, K5_THREADS, 0, h->stream>>>(tel, count, index_base, prior, h->d_partials, h->d_ticket, best_out);
+    return check_launch(h);
+}
+
+i64 neighbourhood_size(int n, int nb, i64 samples) {
+    const i64 nsw = (i64)n * (n - 1) / 2;
+    return nb == SCHED_NBHD_SWAP ? nsw : nb == SCHED_NBHD_SWAP_INSERT ? nsw + (i64)n * (n - 1) : samples;
+}
+
+int read_status(sched_ctx* h) {
+    int* hp = (int*)h->h_pinned;
+    KV_CUDA(cudaMemcpyAsync(hp, h->d_status, sizeof(int), cudaMemcpyDeviceToHost, h->stream));
+    KV_CUDA(cudaStreamSynchronize(h->stream));
+    if (*hp != KV_DEV_OK) {
+        cudaMemsetAsync(h->d_status, 0, sizeof(int), h->stream);
+        return SCHED_E_INTERNAL;
+    }
+    return SCHED_OK;
+}
+
+bool is_permutation(const int32_t* a, int n, std::vector<unsigned char>& seen) {
+    seen.assign(n, 0);
+    for (int q = 0; q < n; ++q) {
+        int v = a[q];
+        if (v < 0 || v >= n || seen[v]) return false;
+        seen[v] = 1;
+    }
+    return true;
+}
+
+}  // namespace
+
+extern "C" {
+
+int sched_init(sched_handle* out, int32_t n, const int32_t* s, const int32_t* o, int64_t M) {
+    return create_common(out, 1, n, s, o, M);
+}
+
+int sched_init_batch(sched_handle* out, int32_t B, int32_t n_each, const int32_t* s, const int32_t* o, int64_t M) {
+    if (n_each > 1024) return SCHED_E_UNSUPPORTED;
+    int rc = create_common(out, B, n_each, s, o, M);
+    if (rc == SCHED_OK) (*out)->batch_handle = true;
+    return rc;
+}
+
+int sched_set_stream(sched_handle h, void* cuda_stream) {
+    KV_ENTER(h);
+    KV_CUDA(cudaStreamSynchronize(h->stream));
+    h->stream = cuda_stream ? (cudaStream_t)cuda_stream : h->own_stream;
+    return SCHED_OK;
+}
+
+int sched_sync(sched_handle h) {
+    KV_ENTER(h);
+    return read_status(h);
+}
+
+int sched_set_base_order(sched_handle h, const int32_t* order) {
+    KV_ENTER(h);
+    if (h->batch_handle || !order) return SCHED_E_INVAL;
+    std::vector<unsigned char> seen;
+    if (!is_permutation(order, h->n, seen)) return SCHED_E_NOT_PERMUTATION;
+    KV_CUDA(cudaMemcpyAsync(h->d_order, order, (size_t)h->n * sizeof(int), cudaMemcpyHostToDevice, h->stream));
+    KV_CUDA(cudaStreamSynchronize(h->stream));
+    h->base_ready = false;
+    return SCHED_OK;
+}
+
+int sched_get_base_order(sched_handle h, int32_t* order_out) {
+    KV_ENTER(h);
+    if (h->batch_handle || !order_out) return SCHED_E_INVAL;
+    KV_CUDA(cudaMemcpyAsync(order_out, h->d_order, (size_t)h->n * sizeof(int), cudaMemcpyDeviceToHost, h->stream));
+    KV_CUDA(cudaStreamSynchronize(h->stream));
+    return SCHED_OK;
+}
+
+int sched_eval_batch_dev(sched_handle h, int kind, int64_t count, const void* candidates,
+                         int64_t* tel_out, uint8_t* feasible_out, int32_t* starts_out) {
+    KV_ENTER(h);
+    if (count < 0 || !tel_out || (count > 0 && !candidates)) return SCHED_E_INVAL;
+    if (count == 0) return SCHED_OK;
+    if (count >= (1ll << 31)) return SCHED_E_UNSUPPORTED;
+    const int n = h->n;
+    if (kind == SCHED_CAND_POLICY) {
+        const size_t smem = (size_t)(n + 1) * 16 + (size_t)n * 8 + (size_t)n * 16 + (size_t)(n + 2) * 4 + (size_t)h->L * 4;
+        if (smem > (size_t)h->smem_optin - 1024) return SCHED_E_UNSUPPORTED;
+        const i64 ctas = (i64)h->B * count;
+        if (ctas >= (1ll << 31)) return SCHED_E_UNSUPPORTED;
+        k3_eval_policy<<<(unsigned)ctas, 32, smem, h->stream>>>(h->d_s, h->d_o, n, h->L, (int)h->M,
+                                                                  (const int*)candidates, (int)count,
+                                                                  (i64*)tel_out, starts_out, h->d_status);
+        KV_TRY(check_launch(h));
+        h->evaluations += ctas;
+        if (feasible_out) KV_CUDA(cudaMemsetAsync(feasible_out, 1, (size_t)ctas, h->stream));
+        return SCHED_OK;
+    }
+    if (h->batch_handle) return SCHED_E_INVAL;
+    if (kind == SCHED_CAND_MOVE) {
+        KV_TRY(launch_moves(h, 0, (const i64*)candidates, 0, 0, 0, count, (i64*)tel_out, starts_out));
+        if (feasible_out) KV_CUDA(cudaMemsetAsync(feasible_out, 1, (size_t)count, h->stream));
+        return SCHED_OK;
+    }
+    if (kind == SCHED_CAND_ORDER) {
+        OrderEvalParams p;
+        memset(&p, 0, sizeof(p));
+        bool in_smem; unsigned tb;
+        const size_t smem = k3_smem_bytes(h, &in_smem, &tb);
+        p.n = n; p.L = h->L; p.M = (int)h->M; p.tbl_id = h->d_tbl_id;
+        p.table_in_smem = in_smem ? 1 : 0; p.table_bytes = tb;
+        p.orders = (const int*)candidates; p.count = count; p.tel_out = (i64*)tel_out; p.starts_out = starts_out;
+        p.counter = h->d_counter; p.status = h->d_status;
+        KV_CUDA(cudaMemsetAsync(h->d_counter, 0, sizeof(unsigned), h->stream));
+        k3_eval_orders<<<k3_grid(h, count), K3_THREADS, smem, h->stream>>>(p);
+        KV_TRY(check_launch(h));
+        h->evaluations += count;
+        if (feasible_out) KV_CUDA(cudaMemsetAsync(feasible_out, 1, (size_t)count, h->stream));
+        return SCHED_OK;
+    }
+    if (kind == SCHED_CAND_START_TIMES) {
+        if (starts_out) return SCHED_E_INVAL;
+        const i64 total = count * n;
+        if (total >= (1ll << 31)) return SCHED_E_UNSUPPORTED;
+        // ids of every candidate by ascending (start, id): K1 with one segment per candidate
+        const size_t need = (size_t)total * (2 * sizeof(u64) + 2 * sizeof(int)) + (size_t)(count + 1) * sizeof(int) + 64;
+        if (h->sort_cap < need) {
+            if (h->d_sort) { cudaFree(h->d_sort); h->d_sort = nullptr; h->sort_cap = 0; }
+            KV_CUDA(cudaMalloc(&h->d_sort, need));
+            h->sort_cap = need;
+        }
+        u64* ka = (u64*)h->d_sort; u64* kb = ka + total;
+        int* va = (int*)(kb + total); int* vb = va + total; int* seg = vb + total;
+        k1_keys_start_then_id<<<(unsigned)((total + 255) / 256), 256, 0, h->stream>>>((const int*)candidates, n, total, ka, va, seg, (int)count);
+        KV_TRY(check_launch(h));
+        const unsigned mask = key_byte_mask(bits_of((u64)n), 31);
+        k1_radix_sort_segments<<<(unsigned)(count < 65535 ? count : 65535), K1_THREADS, 0, h->stream>>>(ka, va, kb, vb, seg, nullptr, (int)count, mask);
+        KV_TRY(check_launch(h));
+        StartsEvalParams p;
+        memset(&p, 0, sizeof(p));
+        p.n = n; p.L = h->L; p.M = (int)h->M; p.tbl_id = h->d_tbl_id;
+        p.starts = (const int*)candidates; p.sorted_ids = va; p.count = count;
+        p.tel_out = (i64*)tel_out; p.feasible_out = feasible_out; p.counter = h->d_counter;
+        KV_CUDA(cudaMemsetAsync(h->d_counter, 0, sizeof(unsigned), h->stream));
+        k3_check_starts<<<k3_grid(h, count), K3_THREADS, (size_t)K3_WARPS * h->L * sizeof(int), h->stream>>>(p);
+        KV_TRY(check_launch(h));
+        h->evaluations += count;
+        return SCHED_OK;
+    }
+    return SCHED_E_INVAL;
+}
+
+int sched_eval_batch(sched_handle h, int kind, int64_t count, const void* candidates,
+                     int64_t* tel_out, uint8_t* feasible_out, int32_t* starts_out) {
+    KV_ENTER(h);
+    if (count < 0 || !tel_out || (count > 0 && !candidates)) return SCHED_E_INVAL;
+    if (count == 0) return SCHED_OK;
+    const int n = h->n;
+    size_t cand_bytes = 0; i64 outs = count;
+    if (kind == SCHED_CAND_ORDER) {
+        if (h->batch_handle) return SCHED_E_INVAL;
+        std::vector<unsigned char> seen;
+        for (i64 c = 0; c < count; ++c)
+            if (!is_permutation((const int32_t*)candidates + c * n, n, seen)) return SCHED_E_NOT_PERMUTATION;
+        cand_bytes = (size_t)count * n * sizeof(int);
+    } else if (kind == SCHED_CAND_MOVE) {
+        if (h->batch_handle || n < 2) return SCHED_E_INVAL;
+        const i64 total = neighbourhood_size(n, SCHED_NBHD_SWAP_INSERT, 0);
+        for (i64 c = 0; c < count; ++c) {
+            i64 code = ((const i64*)candidates)[c];
+            if (code < 0 || code >= total) return SCHED_E_INVAL;
+        }
+        cand_bytes = (size_t)count * sizeof(i64);
+    } else if (kind == SCHED_CAND_START_TIMES) {
+        if (h->batch_handle || starts_out) return SCHED_E_INVAL;
+        for (i64 k = 0; k < count * n; ++k) {
+            int v = ((const int32_t*)candidates)[k];
+            if (v < 0 || v >= (1 << 30)) return SCHED_E_INVAL;
+        }
+        cand_bytes = (size_t)count * n * sizeof(int);
+    } else if (kind == SCHED_CAND_POLICY) {
+        for (i64 c = 0; c < count; ++c) {
+            int v = ((const int32_t*)candidates)[c];
+            if (v < SCHED_POLICY_FCFS || v > SCHED_POLICY_SORTED_F) return SCHED_E_INVAL;
+        }
+        cand_bytes = (size_t)count * sizeof(int);
+        outs = (i64)h->B * count;
+    } else {
+        return SCHED_E_INVAL;
+    }
+    // staging layout: candidates | tel | feasible | starts
+    const size_t off_tel = (cand_bytes + 255) & ~(size_t)255;
+    const size_t off_feas = off_tel + (((size_t)outs * sizeof(i64) + 255) & ~(size_t)255);
+    const size_t off_starts = off_feas + (((size_t)outs + 255) & ~(size_t)255);
+    const size_t starts_bytes = starts_out ? (size_t)outs * n * sizeof(int) : 0;
+    KV_TRY(ensure_stage(h, off_starts + starts_bytes + 256));
+    char* base = (char*)h->d_stage;
+    KV_CUDA(cudaMemcpyAsync(base, candidates, cand_bytes, cudaMemcpyHostToDevice, h->stream));
+    int rc = sched_eval_batch_dev(h, kind, count, base, (int64_t*)(base + off_tel),
+                                  feasible_out ? (uint8_t*)(base + off_feas) : nullptr,
+                                  starts_out ? (int32_t*)(base + off_starts) : nullptr);
+    if (rc != SCHED_OK) { cudaStreamSynchronize(h->stream); return rc; }
+    KV_CUDA(cudaMemcpyAsync(tel_out, base + off_tel, (size_t)outs * sizeof(i64), cudaMemcpyDeviceToHost, h->stream));
+    if (feasible_out) KV_CUDA(cudaMemcpyAsync(feasible_out, base + off_feas, (size_t)outs, cudaMemcpyDeviceToHost, h->stream));
+    if (starts_out) KV_CUDA(cudaMemcpyAsync(starts_out, base + off_starts, starts_bytes, cudaMemcpyDeviceToHost, h->stream));
+    return read_status(h);
+}
+
+int sched_sweep_dev(sched_handle h, int sampled, uint64_t seed, int32_t iteration,
+                    int64_t first_code, int64_t count, int64_t* tel_out, int64_t* best_out) {
+    KV_ENTER(h);
+    if (h->batch_handle || h->n < 2 || count <= 0 || first_code < 0 || !best_out) return SCHED_E_INVAL;
+    if (!sampled && first_code + count > neighbourhood_size(h->n, SCHED_NBHD_SWAP_INSERT, 0)) return SCHED_E_INVAL;
+    i64* tel = (i64*)tel_out;
+    for (i64 done = 0; done < count; done += kSweepChunk) {
+        const i64 c = count - done < kSweepChunk ? count - done : kSweepChunk;
+        i64* dst;
+        if (tel) dst = tel + done;
+        else { KV_TRY(ensure_tel(h, c)); dst = h->d_tel; }
+        KV_TRY(launch_moves(h, sampled ? 2 : 1, nullptr, first_code + done, seed, iteration, c, dst, nullptr));
+        KV_TRY(launch_argmin(h, dst, c, first_code + done, done ? (const i64*)best_out : nullptr, (i64*)best_out));
+    }
+    return SCHED_OK;
+}
+
+int sched_sorted_f_dev(sched_handle h, int32_t* order_out, int32_t* batch_offsets_out,
+                       int32_t* num_batches_out, int64_t* tel_out) {
+    KV_ENTER(h);
+    if (h->batch_handle) return SCHED_E_INVAL;
+    const int n = h->n;
+    cudaStream_t st = h->stream;
+    // S1: ascending (s+o, o, index)
+    k1_keys_total_size<<<(n + 255) / 256, 256, 0, st>>>(h->d_s, h->d_o, n, h->d_keys_a, h->d_vals_a, SCHED_POLICY_SORTED_F);
+    KV_TRY(check_launch(h));
+    k1_radix_sort_segments<<<1, K1_THREADS, 0, st>>>(h->d_keys_a, h->d_vals_a, h->d_keys_b, h->d_vals_b, h->d_seg_off, nullptr, 1,
+                                                      key_byte_mask(bits_of((u64)h->omax), bits_of((u64)h->M)));
+    KV_TRY(check_launch(h));
+    // S2: prefix sums + F-metric batch boundaries
+    k2_prefix_f<<<1, 1024, 0, st>>>(h->d_s, h->d_o, h->d_vals_a, n, h->M, h->d_prefP, h->d_prefO, h->d_batch_off, h->d_num_batches);
+    KV_TRY(check_launch(h));
+    // each batch by ascending (o, index)
+    k1_keys_output_then_id<<<(n + 255) / 256, 256, 0, st>>>(h->d_o, h->d_vals_a, n, h->d_keys_a, h->d_vals_a);
+    KV_TRY(check_launch(h));
+    int grid = n < 4 * h->sm_count ? n : 4 * h->sm_count;
+    k1_radix_sort_segments<<<grid, K1_THREADS, 0, st>>>(h->d_keys_a, h->d_vals_a, h->d_keys_b, h->d_vals_b, h->d_batch_off, h->d_num_batches, 0,
+                                                         key_byte_mask(bits_of((u64)n), bits_of((u64)h->omax)));
+    KV_TRY(check_launch(h));
+    KV_CUDA(cudaMemcpyAsync(h->d_order, h->d_vals_a, (size_t)n * sizeof(int), cudaMemcpyDeviceToDevice, st));
+    h->base_ready = false;
+    KV_TRY(ensure_base(h));
+    if (order_out) KV_CUDA(cudaMemcpyAsync(order_out, h->d_order, (size_t)n * sizeof(int), cudaMemcpyDeviceToDevice, st));
+    if (batch_offsets_out) KV_CUDA(cudaMemcpyAsync(batch_offsets_out, h->d_batch_off, (size_t)(n + 1) * sizeof(int), cudaMemcpyDeviceToDevice, st));
+    if (num_batches_out) KV_CUDA(cudaMemcpyAsync(num_batches_out, h->d_num_batches, sizeof(int), cudaMemcpyDeviceToDevice, st));
+    if (tel_out) KV_CUDA(cudaMemcpyAsync(tel_out, h->d_base_tel, sizeof(i64), cudaMemcpyDeviceToDevice, st));
+    return SCHED_OK;
+}
+
+int sched_sorted_f(sched_handle h, int32_t* order_out, int32_t* batch_offsets_out,
+                   int32_t* num_batches_out, int64_t* tel_out) {
+    KV_ENTER(h);
+    KV_TRY(sched_sorted_f_dev(h, nullptr, nullptr, nullptr, nullptr));
+    const int n = h->n;
+    cudaStream_t st = h->stream;
+    int nb = 0;
+    KV_CUDA(cudaMemcpyAsync(&nb, h->d_num_batches, sizeof(int), cudaMemcpyDeviceToHost, st));
+    if (order_out) KV_CUDA(cudaMemcpyAsync(order_out, h->d_order, (size_t)n * sizeof(int), cudaMemcpyDeviceToHost, st));
+    if (tel_out) KV_CUDA(cudaMemcpyAsync(tel_out, h->d_base_tel, sizeof(i64), cudaMemcpyDeviceToHost, st));
+    KV_CUDA(cudaStreamSynchronize(st));
+    if (num_batches_out) *num_batches_out = nb;
+    if (batch_offsets_out) {
+        KV_CUDA(cudaMemcpyAsync(batch_offsets_out, h->d_batch_off, (size_t)(nb + 1) * sizeof(int), cudaMemcpyDeviceToHost, st));
+    }
+    return read_status(h);
+}
+
+int sched_local_search(sched_handle h, int neighbourhood, int32_t iters, uint64_t seed,
+                       int64_t samples_per_iter, int32_t* order_inout, int64_t* tel_out,
+                       int32_t* iters_done_out, int64_t* trace_out) {
+    KV_ENTER(h);
+    if (h->batch_handle || iters < 0) return SCHED_E_INVAL;
+    if (neighbourhood < SCHED_NBHD_SWAP || neighbourhood > SCHED_NBHD_SAMPLED) return SCHED_E_INVAL;
+    if (neighbourhood == SCHED_NBHD_SAMPLED && samples_per_iter < 1) return SCHED_E_INVAL;
+    const int n = h->n;
+    if (order_inout) KV_TRY(sched_set_base_order(h, order_inout));
+    cudaStream_t st = h->stream;
+    const int sampled = neighbourhood == SCHED_NBHD_SAMPLED ? 1 : 0;
+    const i64 total = n >= 2 ? neighbourhood_size(n, neighbourhood, samples_per_iter) : 0;
+    KV_TRY(ensure_base(h));
+    i64* d_cur = (i64*)h->d_state;               // {current TEL, accepted flag}
+    int* d_acc = (int*)(d_cur + 1);
+    KV_CUDA(cudaMemcpyAsync(d_cur, h->d_base_tel, sizeof(i64), cudaMemcpyDeviceToDevice, st));
+    i64* hp = (i64*)h->h_pinned;                 // {best TEL, best code, accepted, base TEL}
+    int it = 0;
+    i64 cur_tel = 0;
+    KV_CUDA(cudaMemcpyAsync(&hp[3], h->d_base_tel, sizeof(i64), cudaMemcpyDeviceToHost, st));
+    KV_CUDA(cudaStreamSynchronize(st));
+    cur_tel = hp[3];
+    for (; it < iters && total > 0; ++it) {
+        KV_TRY(ensure_tel(h, total < kSweepChunk ? total : kSweepChunk));
+        for (i64 done = 0; done < total; done += kSweepChunk) {
+            const i64 c = total - done < kSweepChunk ? total - done : kSweepChunk;
+            KV_TRY(launch_moves(h, sampled ? 2 : 1, nullptr, done, seed, it, c, h->d_tel, nullptr));
+            KV_TRY(launch_argmin(h, h->d_tel, c, done, done ? h->d_best : nullptr, h->d_best));
+        }
+        k5_accept_move<<<1, 256, 0, st>>>(h->d_order, n, h->d_best, d_cur, d_acc, h->d_vals_b, sampled, seed, it);
+        KV_TRY(check_launch(h));
+        KV_CUDA(cudaMemcpyAsync(&hp[0], h->d_best, 2 * sizeof(i64), cudaMemcpyDeviceToHost, st));
+        KV_CUDA(cudaMemcpyAsync(&hp[2], d_acc, sizeof(int), cudaMemcpyDeviceToHost, st));
+        KV_CUDA(cudaStreamSynchronize(st));
+        if (trace_out) { trace_out[2 * it] = hp[1]; trace_out[2 * it + 1] = hp[0]; }
+        const bool accepted = *(int*)&hp[2] != 0;
+        if (accepted) {
+            cur_tel = hp[0];
+            h->base_ready = false;
+            KV_TRY(ensure_base(h));
+            // the re-simulated base order must reproduce the TEL that won the sweep
+            KV_CUDA(cudaMemcpyAsync(&hp[3], h->d_base_tel, sizeof(i64), cudaMemcpyDeviceToHost, st));
+            KV_CUDA(cudaStreamSynchronize(st));
+            if (hp[3] != cur_tel) return SCHED_E_INTERNAL;
+        } else if (!sampled) {
+            ++it;
+            break;
+        }
+    }
+    if (order_inout) KV_CUDA(cudaMemcpyAsync(order_inout, h->d_order, (size_t)n * sizeof(int), cudaMemcpyDeviceToHost, st));
+    if (tel_out) *tel_out = cur_tel;
+    if (iters_done_out) *iters_done_out = it;
+    return read_status(h);
+}
+
+int sched_stats(sched_handle h, int64_t* kernel_launches_out, int64_t* evaluations_out) {
+    if (!h) return SCHED_E_INVAL;
+    if (kernel_launches_out) *kernel_launches_out = h->launches;
+    if (evaluations_out) *evaluations_out = h->evaluations;
+    return SCHED_OK;
+}
+
+int sched_destroy(sched_handle h) {
+    if (!h) return SCHED_E_INVAL;
+    DeviceGuard guard(h->device);
+    cudaStreamSynchronize(h->stream);
+    free_ctx(h);
+    return SCHED_OK;
+}
+
+const char* sched_strerror(int code) {
+    switch (code) {
+        case SCHED_OK: return "ok";
+        case SCHED_E_INVAL: return "invalid argument";
+        case SCHED_E_NOT_PERMUTATION: return "candidate is not a permutation of 0..n-1";
+        case SCHED_E_CUDA: return "CUDA runtime error";
+        case SCHED_E_NOMEM: return "out of memory";
+        case SCHED_E_INTERNAL: return "a bounded device loop hit its cap";
+        case SCHED_E_UNSUPPORTED: return "size not supported by this build";
+        default: return "unknown error code";
+    }
+}
+
+const char* sched_last_cuda_error(void) { return g_last_cuda_error; }
+
+}  // extern "C"

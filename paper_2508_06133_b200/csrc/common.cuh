@@ -1,0 +1,150 @@
+// Shared declarations of the kvsched GPU library: handle layout, error helpers, small device
+// utilities.  Everything here is integer arithmetic; nothing is shared with the CPU checker.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/kvsched.h"
+
+typedef long long i64;
+typedef unsigned long long u64;
+
+#define KV_WARP 32
+#define KV_FULL 0xffffffffu
+
+// Device-side status word (ctx->d_status[0]); non-zero means a bounded loop gave up.
+enum { KV_DEV_OK = 0, KV_DEV_LOOP_CAP = 1, KV_DEV_TMA_TIMEOUT = 2 };
+
+struct SnapHeader {          // simulator state in front of one list position (16 bytes)
+    int t;                   // current round index (number of completed rounds = next start time)
+    int hz;                  // first round after which the timeline is all zero
+    int tel_lo, tel_hi;      // TEL of the positions before this one
+};
+
+struct sched_ctx {
+    int device;
+    cudaStream_t stream, own_stream;
+    int B, n;                // instances, requests per instance
+    i64 M;
+    int omax;                // largest decode length over all instances
+    int L;                   // ring length in cells (multiple of 4, >= omax + 8)
+    i64 sum_o_max;           // largest sum of o over instances (bounds every start time)
+    int sm_count;
+    int smem_optin;          // max dynamic shared memory per block (bytes)
+
+    int *d_s, *d_o;          // [B*n]
+    int2* d_tbl_id;          // (s, o) by request id [B*n]
+    int2* d_tbl_base;        // (s, o) by base position [n]
+    int* d_order;            // base order [n]
+    bool base_ready;         // d_tbl_base + snapshots match d_order
+    bool batch_handle;       // created by sched_init_batch
+    int* d_base_starts;      // start of every position of the base order [n]
+    i64* d_state;            // local-search state {current TEL, accepted flag}
+    void* h_pinned;          // 64 bytes of pinned host memory for small read-backs
+    void* d_sort;            // grow-only scratch for sorting explicit start times
+    size_t sort_cap;
+
+    // snapshots of the base run
+    int snap_stride, snap_count;
+    int* d_snap_ring;        // [snap_count][L]
+    SnapHeader* d_snap_hdr;  // [snap_count]
+    i64* d_base_tel;         // [1]
+
+    // scratch
+    unsigned int* d_counter; // work counter(s)
+    int* d_status;           // [1] device status
+    i64* d_tel;              // [tel_cap] per-candidate TEL scratch
+    i64 tel_cap;
+    i64* d_best;             // [2] (TEL, index) + partials
+    i64* d_partials;         // [2 * max_blocks]
+    unsigned int* d_ticket;  // [1]
+
+    // sort / F-metric scratch (single-instance handles)
+    u64 *d_keys_a, *d_keys_b;
+    int *d_vals_a, *d_vals_b;
+    i64 *d_prefP, *d_prefO;  // [n+1]
+    int* d_batch_off;        // [n+1]
+    int* d_num_batches;      // [1]
+    int* d_seg_off;          // [2] offsets {0, n} for whole-array sorts
+
+    // staging for the host-pointer entry points
+    void* d_stage;
+    size_t stage_cap;
+
+    i64 launches, evaluations;
+};
+
+extern thread_local char g_last_cuda_error[256];
+int kv_cuda_fail(cudaError_t e, const char* what);
+
+#define KV_CUDA(expr)                                                        \
+    do {                                                                     \
+        cudaError_t e__ = (expr);                                            \
+        if (e__ != cudaSuccess) return kv_cuda_fail(e__, #expr);             \
+    } while (0)
+
+#define KV_TRY(expr)                                                         \
+    do {                                                                     \
+        int rc__ = (expr);                                                   \
+        if (rc__ != SCHED_OK) return rc__;                                   \
+    } while (0)
+
+// ------------------------------------------------------------------------------------ device utils
+__device__ __forceinline__ int kv_lane() { return threadIdx.x & 31; }
+
+__device__ __forceinline__ int kv_warp_max(int v) { return __reduce_max_sync(KV_FULL, v); }
+__device__ __forceinline__ int kv_warp_min(int v) { return __reduce_min_sync(KV_FULL, v); }
+
+// splitmix64 step, used by the sampled neighbourhood (published generator by Steele, Lea, Flood).
+__host__ __device__ __forceinline__ u64 kv_mix64(u64 z) {
+    z += 0x9E3779B97F4A7C15ull;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
+}
+
+struct Move { int type, i, j; };     // type 0 = swap (i < j), 1 = insert i -> j, -1 = identity
+
+// Move code -> (type, i, j).  Swaps are numbered row by row: row i holds n-1-i codes and starts at
+// i*(2n-i-1)/2.  The row is first guessed from a square root and then corrected with exact integer
+// comparisons, so the result does not depend on floating-point rounding.
+__host__ __device__ __forceinline__ Move kv_decode_move(int n, i64 code) {
+    Move m;
+    i64 nsw = (i64)n * (n - 1) / 2;
+    if (code < nsw) {
+        double b = 2.0 * n - 1.0;
+        i64 i = (i64)((b - sqrt(b * b - 8.0 * (double)code)) * 0.5);
+        if (i < 0) i = 0;
+        if (i > n - 2) i = n - 2;
+        while (i > 0 && i * (2 * (i64)n - i - 1) / 2 > code) --i;
+        while ((i + 1) * (2 * (i64)n - (i + 1) - 1) / 2 <= code) ++i;
+        m.type = 0; m.i = (int)i; m.j = (int)(i + 1 + (code - i * (2 * (i64)n - i - 1) / 2));
+    } else {
+        i64 c = code - nsw;
+        int i = (int)(c / (n - 1)), r = (int)(c % (n - 1));
+        m.type = 1; m.i = i; m.j = r < i ? r : r + 1;
+    }
+    return m;
+}
+
+__host__ __device__ __forceinline__ Move kv_sample_move(int n, u64 seed, int it, i64 mcount) {
+    u64 h1 = kv_mix64(seed ^ kv_mix64(((u64)(uint32_t)it << 32) + (u64)mcount));
+    u64 h2 = kv_mix64(h1);
+    Move m;
+    m.type = (int)(h1 & 1);
+    m.i = (int)((h1 >> 1) % (u64)n);
+    m.j = (int)(((u64)m.i + 1 + h2 % (u64)(n - 1)) % (u64)n);
+    if (m.type == 0 && m.i > m.j) { int x = m.i; m.i = m.j; m.j = x; }
+    return m;
+}
+
+// Position q of the moved order -> position in the base order.
+__host__ __device__ __forceinline__ int kv_map_pos(const Move& m, int q) {
+    if (m.type == 0) return q == m.i ? m.j : (q == m.j ? m.i : q);
+    if (m.type == 1) {
+        if (m.i < m.j) return (q < m.i || q > m.j) ? q : (q == m.j ? m.i : q + 1);
+        return (q < m.j || q > m.i) ? q : (q == m.j ? m.i : q - 1);
+    }
+    return q;
+}

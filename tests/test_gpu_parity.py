@@ -1,0 +1,299 @@
+"""GPU parity: every integer the CUDA library returns equals the CPU oracle's on the same inputs.
+
+All calls go through the C-ABI (``binding.Scheduler`` only marshals arguments).  Bit-exact: TELs,
+start times, feasibility flags, Sorted-F orders and batch boundaries, local-search traces.
+"""
+import numpy as np
+import pytest
+
+import oracle as orc
+from paper_2508_06133_b200 import binding as kv
+from paper_2508_06133_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+def rand_instance(rng, n, M, smax, omax):
+    s = rng.integers(1, smax + 1, n).astype(np.int32)
+    o = rng.integers(1, omax + 1, n).astype(np.int32)
+    bad = s.astype(np.int64) + o > M
+    s[bad] = 1
+    return s, o
+
+
+def all_codes(n, inserts=True):
+    return np.arange(n * (n - 1) // 2 + (n * (n - 1) if inserts else 0), dtype=np.int64)
+
+
+def oracle_moves(s, o, M, base, codes):
+    mv = [orc.decode_move(len(s), int(c)) for c in codes]
+    return orc.eval_moves(s, o, M, base, [m[0] for m in mv], [m[1] for m in mv], [m[2] for m in mv])
+
+
+# ------------------------------------------------------------------------------------ ORDER
+def test_orders_small_random_instances_tel_and_starts():
+    rng = np.random.default_rng(1)
+    for trial in range(60):
+        n = int(rng.integers(1, 70))
+        M = int(rng.integers(8, 300))
+        s, o = rand_instance(rng, n, M, max(1, M // 2), max(1, M // 3))
+        orders = np.stack([rng.permutation(n) for _ in range(9)]).astype(np.int32)
+        with kv.Scheduler(s, o, M) as h:
+            tel, feas, starts = h.eval_batch(kv.CAND_ORDER, orders, want_feasible=True, want_starts=True)
+        assert feas.all()
+        for c in range(len(orders)):
+            p, t, _ = orc.list_schedule_alg1(s, o, M, orders[c])
+            assert tel[c] == t
+            assert (starts[c] == p).all()
+
+
+def test_orders_paper_example_and_closed_form(golden):
+    s = np.array([63] + [1] * 21, dtype=np.int32)
+    o = np.array([1] + [2] * 21, dtype=np.int32)
+    orders = np.stack([np.arange(22), np.array(list(range(1, 22)) + [0])]).astype(np.int32)
+    with kv.Scheduler(s, o, 64) as h:
+        tel, _, _ = h.eval_batch(kv.CAND_ORDER, orders)
+    assert tel.tolist() == [golden["example1_tel_mcsf"], golden["example1_tel_sortedf"]]
+    M = 6561
+    s = np.array([80] * M + [1] * 59049, dtype=np.int32)
+    o = np.array([1] * M + [2] * 59049, dtype=np.int32)
+    with kv.Scheduler(s, o, M) as h:
+        tel, _, _ = h.eval_batch(kv.CAND_ORDER, np.arange(len(s), dtype=np.int32)[None, :])
+    assert tel[0] == golden["thm1_M6561_tel_mcsf"]
+
+
+def test_orders_long_waits_and_ring_wrap():
+    """Few huge requests force waits longer than a decode length; tiny o_max wraps the ring often."""
+    rng = np.random.default_rng(2)
+    for omax, M in ((1, 50), (2, 40), (3, 64), (40, 100), (200, 1000)):
+        n = 120
+        s = rng.integers(1, M - omax, n).astype(np.int32)
+        o = rng.integers(1, omax + 1, n).astype(np.int32)
+        s[::7] = M - o[::7]                                  # requests that need the machine alone
+        orders = np.stack([rng.permutation(n) for _ in range(5)]).astype(np.int32)
+        with kv.Scheduler(s, o, M) as h:
+            tel, _, starts = h.eval_batch(kv.CAND_ORDER, orders, want_starts=True)
+        for c in range(5):
+            p, t, _ = orc.list_schedule_rounds(s, o, M, orders[c])
+            assert tel[c] == t and (starts[c] == p).all()
+
+
+def test_orders_mixed_1k():
+    inst = W.mixed_1k()
+    orders = W.random_permutations(inst.n, 6, seed=9)
+    orders[0] = orc.policy_order(inst.s, inst.o, orc.SHORTEST_OUTPUT_FIRST)
+    orders[1] = orc.policy_order(inst.s, inst.o, orc.TOTAL_SIZE_FIRST)
+    with kv.Scheduler(inst.s, inst.o, inst.M) as h:
+        tel, _, starts = h.eval_batch(kv.CAND_ORDER, orders, want_starts=True)
+    for c in range(len(orders)):
+        p, t, _ = orc.list_schedule_rounds(inst.s, inst.o, inst.M, orders[c])
+        assert tel[c] == t and (starts[c] == p).all()
+    p, t, _ = orc.list_schedule_alg1(inst.s, inst.o, inst.M, orders[1])      # literal Algorithm 1 once
+    assert tel[1] == t
+
+
+# ------------------------------------------------------------------------------------ MOVE
+def test_moves_full_neighbourhood_tiny_backlog():
+    inst = W.tiny()
+    base, _ = orc.sorted_f_prefix(inst.s, inst.o, inst.M)
+    codes = all_codes(inst.n)
+    with kv.Scheduler(inst.s, inst.o, inst.M) as h:
+        h.set_base_order(base)
+        tel, _, starts = h.eval_batch(kv.CAND_MOVE, codes, want_starts=True)
+    ref = oracle_moves(inst.s, inst.o, inst.M, base, codes)
+    assert (tel == ref).all()
+    for c in (0, 5, 119, 120, 200, len(codes) - 1):
+        cand = orc.apply_move(base, *orc.decode_move(inst.n, int(codes[c])))
+        assert (starts[c] == orc.list_schedule_alg1(inst.s, inst.o, inst.M, cand)[0]).all()
+
+
+def test_moves_random_small_instances_all_codes():
+    rng = np.random.default_rng(3)
+    for trial in range(25):
+        n = int(rng.integers(2, 40))
+        M = int(rng.integers(10, 200))
+        s, o = rand_instance(rng, n, M, M // 2, max(1, M // 3))
+        base = rng.permutation(n).astype(np.int32)
+        codes = all_codes(n)
+        with kv.Scheduler(s, o, M) as h:
+            h.set_base_order(base)
+            tel, _, _ = h.eval_batch(kv.CAND_MOVE, codes)
+        assert (tel == oracle_moves(s, o, M, base, codes)).all()
+
+
+def test_moves_sampled_codes_mixed_1k_and_10k():
+    for inst, count in ((W.mixed_1k(), 1500), (W.mixed_10k(), 160)):
+        base, _ = orc.sorted_f_prefix(inst.s, inst.o, inst.M)
+        n = inst.n
+        total = n * (n - 1) // 2 + n * (n - 1)
+        codes = (W.u64(77, 0, np.arange(count)) % np.uint64(total)).astype(np.int64)
+        codes[:4] = [0, n * (n - 1) // 2 - 1, n * (n - 1) // 2, total - 1]
+        with kv.Scheduler(inst.s, inst.o, inst.M) as h:
+            h.set_base_order(base)
+            tel, _, _ = h.eval_batch(kv.CAND_MOVE, codes)
+        assert (tel == oracle_moves(inst.s, inst.o, inst.M, base, codes)).all()
+
+
+# ------------------------------------------------------------------------------------ Sorted-F
+def test_sorted_f_matches_oracle():
+    rng = np.random.default_rng(4)
+    cases = [W.tiny(), W.mixed_1k(), W.mixed_10k(), W.paper_scale()]
+    for trial in range(30):
+        n = int(rng.integers(1, 400))
+        M = int(rng.integers(10, 2000))
+        s, o = rand_instance(rng, n, M, M // 2, max(1, M // 3))
+        cases.append(W.Instance("rand", s, o, M))
+    ties = W.Instance("ties", np.array([3, 3, 1, 5, 3, 1] * 20, dtype=np.int32), np.array([2, 2, 4, 2, 2, 4] * 20, dtype=np.int32), 37)
+    cases.append(ties)
+    for inst in cases:
+        with kv.Scheduler(inst.s, inst.o, inst.M) as h:
+            order, offs, tel = h.sorted_f()
+            assert (h.get_base_order() == order).all()
+        r_order, r_offs = orc.sorted_f_prefix(inst.s, inst.o, inst.M)
+        assert (offs == r_offs).all(), inst.name
+        assert (order == r_order).all(), inst.name
+        assert tel == orc.list_schedule_rounds(inst.s, inst.o, inst.M, r_order)[1]
+
+
+def test_sorted_f_example1(golden):
+    s = np.array([63] + [1] * 21, dtype=np.int32)
+    o = np.array([1] + [2] * 21, dtype=np.int32)
+    with kv.Scheduler(s, o, 64) as h:
+        order, offs, tel = h.sorted_f()
+    assert offs.tolist() == [0, 21, 22] and order[-1] == 0 and tel == golden["example1_tel_sortedf"]
+
+
+# ------------------------------------------------------------------------------------ POLICY
+def test_policy_sweep_small_batch():
+    s, o, M = W.policy_sweep(num_instances=24, n_each=256)
+    pols = np.array([kv.POLICY_SORTED_F, kv.POLICY_FCFS, kv.POLICY_SOF, kv.POLICY_TOTAL_SIZE], dtype=np.int32)
+    with kv.Scheduler.batch(s, o, M) as h:
+        tel, feas, starts = h.eval_batch(kv.CAND_POLICY, pols, want_feasible=True, want_starts=True)
+    assert tel.shape == (24, 4) and feas.all()
+    for b in range(24):
+        refs = [orc.sorted_f_prefix(s[b], o[b], M)[0], orc.policy_order(s[b], o[b], orc.FCFS),
+                orc.policy_order(s[b], o[b], orc.SHORTEST_OUTPUT_FIRST), orc.policy_order(s[b], o[b], orc.TOTAL_SIZE_FIRST)]
+        for k, order in enumerate(refs):
+            p, t, _ = orc.list_schedule_rounds(s[b], o[b], M, order)
+            assert tel[b, k] == t
+            assert (starts[b, k] == p).all()
+
+
+def test_policy_on_single_instance_handle_and_odd_sizes():
+    rng = np.random.default_rng(6)
+    for n in (1, 2, 31, 33, 100):
+        M = 300
+        s, o = rand_instance(rng, n, M, 100, 60)
+        with kv.Scheduler(s, o, M) as h:
+            tel, _, _ = h.eval_batch(kv.CAND_POLICY, np.array([3, 2, 1, 0], dtype=np.int32))
+        refs = [orc.sorted_f_prefix(s, o, M)[0], orc.policy_order(s, o, 2), orc.policy_order(s, o, 1), orc.policy_order(s, o, 0)]
+        assert tel[0].tolist() == [orc.list_schedule_alg1(s, o, M, r)[1] for r in refs]
+
+
+# ------------------------------------------------------------------------------------ START_TIMES
+def test_start_times_checker():
+    rng = np.random.default_rng(7)
+    for trial in range(20):
+        n = int(rng.integers(1, 50))
+        M = int(rng.integers(20, 200))
+        s, o = rand_instance(rng, n, M, M // 2, max(1, M // 4))
+        good = orc.list_schedule_alg1(s, o, M, rng.permutation(n))[0]
+        cands = [good]
+        for _ in range(6):                                 # perturbed starts: some overflow, some do not
+            p = good.copy()
+            k = rng.integers(0, n, max(1, n // 4))
+            p[k] = np.maximum(0, p[k] + rng.integers(-5, 6, len(k)))
+            cands.append(p)
+        cands.append(np.zeros(n, dtype=np.int64))          # everything at once
+        cands.append(good + 1000)                          # far beyond the ring length
+        cands = np.stack(cands).astype(np.int32)
+        with kv.Scheduler(s, o, M) as h:
+            tel, feas, _ = h.eval_batch(kv.CAND_START_TIMES, cands, want_feasible=True)
+        for c in range(len(cands)):
+            r = orc.check_schedule(s, o, M, cands[c])
+            assert tel[c] == r["tel"] and bool(feas[c]) == r["feasible"]
+        assert feas[0] == 1
+
+
+# ------------------------------------------------------------------------------------ local search
+def test_local_search_tiny_backlog_full_swap_sweeps():
+    inst = W.tiny()
+    base, _ = orc.sorted_f_prefix(inst.s, inst.o, inst.M)
+    for nb, onb in ((kv.NBHD_SWAP, orc.SWAP), (kv.NBHD_SWAP_INSERT, orc.SWAP_INSERT)):
+        with kv.Scheduler(inst.s, inst.o, inst.M) as h:
+            final, tel, done, trace = h.local_search(nb, 200, order=base)
+        r_final, r_tel, r_done, r_trace = orc.local_search(inst.s, inst.o, inst.M, onb, 200, base)
+        assert (final == r_final).all() and tel == r_tel and done == r_done
+        assert (trace == r_trace).all()
+
+
+def test_local_search_random_instances_to_local_optimum():
+    rng = np.random.default_rng(8)
+    for trial in range(6):
+        n = int(rng.integers(5, 30))
+        M = int(rng.integers(30, 150))
+        s, o = rand_instance(rng, n, M, M // 2, M // 4)
+        start = rng.permutation(n).astype(np.int32)
+        with kv.Scheduler(s, o, M) as h:
+            final, tel, done, trace = h.local_search(kv.NBHD_SWAP_INSERT, 500, order=start)
+        r_final, r_tel, r_done, r_trace = orc.local_search(s, o, M, orc.SWAP_INSERT, 500, start)
+        assert (final == r_final).all() and tel == r_tel and done == r_done and (trace == r_trace).all()
+
+
+def test_local_search_sampled_and_resume():
+    inst = W.mixed_backlog(400, 21, 30000)
+    base, _ = orc.sorted_f_prefix(inst.s, inst.o, inst.M)
+    r_final, r_tel, r_done, r_trace = orc.local_search(inst.s, inst.o, inst.M, orc.SAMPLED, 4, base, seed=99, samples=300)
+    with kv.Scheduler(inst.s, inst.o, inst.M) as h:
+        h.sorted_f()
+        final, tel, done, trace = h.local_search(kv.NBHD_SAMPLED, 4, seed=99, samples_per_iter=300)
+        assert (final == r_final).all() and tel == r_tel and done == r_done == 4 and (trace == r_trace).all()
+        assert (h.get_base_order() == r_final).all()       # the handle keeps the result: a run can be resumed
+
+
+def test_local_search_first_sweeps_mixed_1k():
+    inst = W.mixed_1k()
+    with kv.Scheduler(inst.s, inst.o, inst.M) as h:
+        base, _, tel0 = h.sorted_f()
+        final, tel, done, trace = h.local_search(kv.NBHD_SWAP, 2)
+    assert done == 2 and tel <= tel0
+    # the accepted moves really have the TELs claimed, and the final order is what they produce
+    cur = base
+    for code, best in trace:
+        cand = orc.apply_move(cur, *orc.decode_move(inst.n, int(code)))
+        assert orc.list_schedule_rounds(inst.s, inst.o, inst.M, cand)[1] == best
+        if best < orc.list_schedule_rounds(inst.s, inst.o, inst.M, cur)[1]:
+            cur = cand
+    assert (final == cur).all()
+    # no sampled neighbour of the first sweep beats the reported best
+    n = inst.n
+    codes = (W.u64(5, 0, np.arange(400)) % np.uint64(n * (n - 1) // 2)).astype(np.int64)
+    assert oracle_moves(inst.s, inst.o, inst.M, base, codes).min() >= trace[0][1]
+
+
+# ------------------------------------------------------------------------------------ errors on a live handle
+def test_error_paths_on_a_handle():
+    s, o = np.array([2, 3, 4], dtype=np.int32), np.array([1, 2, 3], dtype=np.int32)
+    with kv.Scheduler(s, o, 20) as h:
+        with pytest.raises(kv.SchedError) as e:
+            h.eval_batch(kv.CAND_ORDER, np.array([[0, 1, 1]], dtype=np.int32))
+        assert e.value.code == kv.E_NOT_PERMUTATION
+        with pytest.raises(kv.SchedError) as e:
+            h.set_base_order(np.array([0, 1, 3], dtype=np.int32))
+        assert e.value.code == kv.E_NOT_PERMUTATION
+        with pytest.raises(kv.SchedError) as e:
+            h.eval_batch(kv.CAND_MOVE, np.array([9], dtype=np.int64))       # 3 swaps + 6 inserts = codes 0..8
+        assert e.value.code == kv.E_INVAL
+        with pytest.raises(kv.SchedError) as e:
+            h.eval_batch(kv.CAND_POLICY, np.array([7], dtype=np.int32))
+        assert e.value.code == kv.E_INVAL
+        with pytest.raises(kv.SchedError) as e:
+            h.eval_batch(kv.CAND_START_TIMES, np.array([[0, -1, 0]], dtype=np.int32))
+        assert e.value.code == kv.E_INVAL
+        with pytest.raises(kv.SchedError) as e:
+            h.eval_batch(17, np.array([0], dtype=np.int32))
+        assert e.value.code == kv.E_INVAL
+        tel, _, _ = h.eval_batch(kv.CAND_ORDER, np.array([[2, 1, 0]], dtype=np.int32))   # still usable
+        assert tel[0] == orc.list_schedule_alg1(s, o, 20, [2, 1, 0])[1]
+        launches, evals = h.stats()
+        assert launches > 0 and evals >= 1
