@@ -106,7 +106,7 @@ size_t k3_smem_bytes(const sched_ctx* h, bool* table_in_smem, unsigned* table_by
     const size_t rings = (size_t)K3_WARPS * h->L * sizeof(int);
     const unsigned tb = (unsigned)(((size_t)h->n * sizeof(int2) + 15) & ~(size_t)15);
     const size_t with_table = ((size_t)tb + 127) / 128 * 128 + rings;
-    if (with_table <= (size_t)h->smem_optin - 1024) {
+    if (with_table <= (size_t)h->smem_optin - 2048) {
         *table_in_smem = true; *table_bytes = tb; return with_table;
     }
     *table_in_smem = false; *table_bytes = tb; return rings;
@@ -139,7 +139,7 @@ int create_common(sched_ctx** out, int B, int n, const int32_t* s, const int32_t
         h->smem_optin = (int)prop.sharedMemPerBlockOptin;
         h->B = B; h->n = n; h->M = M; h->omax = omax; h->sum_o_max = sum_max;
         h->L = (omax + 8 + 3) & ~3;
-        if ((size_t)K3_WARPS * h->L * sizeof(int) > (size_t)h->smem_optin - 1024) { rc = SCHED_E_UNSUPPORTED; break; }
+        if ((size_t)K3_WARPS * h->L * sizeof(int) > (size_t)h->smem_optin - 2048) { rc = SCHED_E_UNSUPPORTED; break; }
         if (cudaStreamCreateWithFlags(&h->own_stream, cudaStreamNonBlocking) != cudaSuccess) { rc = kv_cuda_fail(cudaGetLastError(), "cudaStreamCreate"); break; }
         h->stream = h->own_stream;
 #define A(call) if ((rc = (call)) != SCHED_OK) break
@@ -183,11 +183,11 @@ int create_common(sched_ctx** out, int B, int n, const int32_t* s, const int32_t
             C(cudaMemcpyAsync(h->d_seg_off, seg, sizeof(seg), cudaMemcpyHostToDevice, st));
         }
         // opt in to large dynamic shared memory once
-        C(cudaFuncSetAttribute(k3_eval_moves, cudaFuncAttributeMaxDynamicSharedMemorySize, h->smem_optin - 1024));
-        C(cudaFuncSetAttribute(k3_eval_orders, cudaFuncAttributeMaxDynamicSharedMemorySize, h->smem_optin - 1024));
-        C(cudaFuncSetAttribute(k3_check_starts, cudaFuncAttributeMaxDynamicSharedMemorySize, h->smem_optin - 1024));
-        C(cudaFuncSetAttribute(k3_eval_policy, cudaFuncAttributeMaxDynamicSharedMemorySize, h->smem_optin - 1024));
-        C(cudaFuncSetAttribute(k3_base_run, cudaFuncAttributeMaxDynamicSharedMemorySize, h->smem_optin - 1024));
+        C(cudaFuncSetAttribute(k3_eval_moves, cudaFuncAttributeMaxDynamicSharedMemorySize, h->smem_optin - 2048));
+        C(cudaFuncSetAttribute(k3_eval_orders, cudaFuncAttributeMaxDynamicSharedMemorySize, h->smem_optin - 2048));
+        C(cudaFuncSetAttribute(k3_check_starts, cudaFuncAttributeMaxDynamicSharedMemorySize, h->smem_optin - 2048));
+        C(cudaFuncSetAttribute(k3_eval_policy, cudaFuncAttributeMaxDynamicSharedMemorySize, h->smem_optin - 2048));
+        C(cudaFuncSetAttribute(k3_base_run, cudaFuncAttributeMaxDynamicSharedMemorySize, h->smem_optin - 2048));
         C(cudaStreamSynchronize(st));       // s, o may be pageable host memory owned by the caller
 #undef C
     } while (0);
@@ -330,7 +330,7 @@ int sched_eval_batch_dev(sched_handle h, int kind, int64_t count, const void* ca
     const int n = h->n;
     if (kind == SCHED_CAND_POLICY) {
         const size_t smem = (size_t)(n + 1) * 16 + (size_t)n * 8 + (size_t)n * 16 + (size_t)(n + 2) * 4 + (size_t)h->L * 4;
-        if (smem > (size_t)h->smem_optin - 1024) return SCHED_E_UNSUPPORTED;
+        if (smem > (size_t)h->smem_optin - 2048) return SCHED_E_UNSUPPORTED;
         const i64 ctas = (i64)h->B * count;
         if (ctas >= (1ll << 31)) return SCHED_E_UNSUPPORTED;
         k3_eval_policy<<<(unsigned)ctas, 32, smem, h->stream>>>(h->d_s, h->d_o, n, h->L, (int)h->M,
