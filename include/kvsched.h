@@ -156,6 +156,11 @@ int sched_local_search(sched_handle h, int neighbourhood, int32_t iters, uint64_
                        int64_t samples_per_iter, int32_t* order_inout, int64_t* tel_out,
                        int32_t* iters_done_out, int64_t* trace_out);
 
+/* Device time, in milliseconds, of the most recent schedule-simulation kernel launch of this handle
+ * (the move / order evaluator), measured with CUDA events recorded on the handle's stream around
+ * that launch.  Waits for the launch to finish.  SCHED_E_INVAL if there was none. */
+int sched_last_eval_kernel_ms(sched_handle h, float* ms_out);
+
 /* Counters since sched_init: kernels launched by this handle, candidates evaluated. */
 int sched_stats(sched_handle h, int64_t* kernel_launches_out, int64_t* evaluations_out);
 

@@ -22,7 +22,7 @@ NBHD_SWAP, NBHD_SWAP_INSERT, NBHD_SAMPLED = 0, 1, 2
 EXPORTS = [
     "sched_init", "sched_init_batch", "sched_set_stream", "sched_sync", "sched_set_base_order",
     "sched_get_base_order", "sched_eval_batch", "sched_eval_batch_dev", "sched_sweep_dev",
-    "sched_sorted_f", "sched_sorted_f_dev", "sched_local_search", "sched_stats", "sched_destroy",
+    "sched_sorted_f", "sched_sorted_f_dev", "sched_local_search", "sched_last_eval_kernel_ms", "sched_stats", "sched_destroy",
     "sched_strerror", "sched_last_cuda_error",
 ]
 
@@ -65,6 +65,7 @@ def load():
     lib.sched_sorted_f_dev.argtypes = [vp, vp, vp, vp, vp]
     lib.sched_local_search.argtypes = [vp, C.c_int, i32, u64, i64, vp, vp, vp, vp]
     lib.sched_stats.argtypes = [vp, vp, vp]
+    lib.sched_last_eval_kernel_ms.argtypes = [vp, vp]
     lib.sched_destroy.argtypes = [vp]
     lib.sched_strerror.argtypes = [C.c_int]
     lib.sched_strerror.restype = C.c_char_p
@@ -150,6 +151,11 @@ class Scheduler:
         a, b = C.c_int64(0), C.c_int64(0)
         _check(load().sched_stats(self._h, C.byref(a), C.byref(b)), "sched_stats")
         return a.value, b.value
+
+    def last_eval_kernel_ms(self):
+        ms = C.c_float(0)
+        _check(load().sched_last_eval_kernel_ms(self._h, C.byref(ms)), "sched_last_eval_kernel_ms")
+        return ms.value
 
     def set_base_order(self, order):
         order = np.ascontiguousarray(order, dtype=np.int32)

@@ -98,6 +98,8 @@ void free_ctx(sched_ctx* h) {
                     h->d_state, h->d_sort};
     for (void* p : ptrs) if (p) cudaFree(p);
     if (h->h_pinned) cudaFreeHost(h->h_pinned);
+    if (h->ev_k3_begin) cudaEventDestroy(h->ev_k3_begin);
+    if (h->ev_k3_end) cudaEventDestroy(h->ev_k3_end);
     if (h->own_stream) cudaStreamDestroy(h->own_stream);
     delete h;
 }
@@ -142,6 +144,7 @@ int create_common(sched_ctx** out, int B, int n, const int32_t* s, const int32_t
         if ((size_t)K3_WARPS * h->L * sizeof(int) > (size_t)h->smem_optin - 2048) { rc = SCHED_E_UNSUPPORTED; break; }
         if (cudaStreamCreateWithFlags(&h->own_stream, cudaStreamNonBlocking) != cudaSuccess) { rc = kv_cuda_fail(cudaGetLastError(), "cudaStreamCreate"); break; }
         h->stream = h->own_stream;
+        if (cudaEventCreate(&h->ev_k3_begin) != cudaSuccess || cudaEventCreate(&h->ev_k3_end) != cudaSuccess) { rc = kv_cuda_fail(cudaGetLastError(), "cudaEventCreate"); break; }
 #define A(call) if ((rc = (call)) != SCHED_OK) break
         A(dev_alloc(&h->d_s, total)); A(dev_alloc(&h->d_o, total));
         A(dev_alloc(&h->d_tbl_id, total + 2));
@@ -234,8 +237,11 @@ int launch_moves(sched_ctx* h, int mode, const i64* codes, i64 first, u64 seed, 
     p.base_order = h->d_order; p.base_starts_pos = h->d_base_starts;
     p.counter = h->d_counter; p.status = h->d_status;
     KV_CUDA(cudaMemsetAsync(h->d_counter, 0, sizeof(unsigned), h->stream));
+    KV_CUDA(cudaEventRecord(h->ev_k3_begin, h->stream));
     k3_eval_moves<<<k3_grid(h, count), K3_THREADS, smem, h->stream>>>(p);
     KV_TRY(check_launch(h));
+    KV_CUDA(cudaEventRecord(h->ev_k3_end, h->stream));
+    h->ev_valid = true;
     h->evaluations += count;
     return SCHED_OK;
 }
@@ -357,8 +363,11 @@ int sched_eval_batch_dev(sched_handle h, int kind, int64_t count, const void* ca
         p.orders = (const int*)candidates; p.count = count; p.tel_out = (i64*)tel_out; p.starts_out = starts_out;
         p.counter = h->d_counter; p.status = h->d_status;
         KV_CUDA(cudaMemsetAsync(h->d_counter, 0, sizeof(unsigned), h->stream));
+        KV_CUDA(cudaEventRecord(h->ev_k3_begin, h->stream));
         k3_eval_orders<<<k3_grid(h, count), K3_THREADS, smem, h->stream>>>(p);
         KV_TRY(check_launch(h));
+        KV_CUDA(cudaEventRecord(h->ev_k3_end, h->stream));
+        h->ev_valid = true;
         h->evaluations += count;
         if (feasible_out) KV_CUDA(cudaMemsetAsync(feasible_out, 1, (size_t)count, h->stream));
         return SCHED_OK;
@@ -571,6 +580,14 @@ int sched_local_search(sched_handle h, int neighbourhood, int32_t iters, uint64_
     if (tel_out) *tel_out = cur_tel;
     if (iters_done_out) *iters_done_out = it;
     return read_status(h);
+}
+
+int sched_last_eval_kernel_ms(sched_handle h, float* ms_out) {
+    KV_ENTER(h);
+    if (!ms_out || !h->ev_valid) return SCHED_E_INVAL;
+    KV_CUDA(cudaEventSynchronize(h->ev_k3_end));
+    KV_CUDA(cudaEventElapsedTime(ms_out, h->ev_k3_begin, h->ev_k3_end));
+    return SCHED_OK;
 }
 
 int sched_stats(sched_handle h, int64_t* kernel_launches_out, int64_t* evaluations_out) {

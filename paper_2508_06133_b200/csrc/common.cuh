@@ -73,6 +73,8 @@ struct sched_ctx {
     size_t stage_cap;
 
     i64 launches, evaluations;
+    cudaEvent_t ev_k3_begin, ev_k3_end;   // around the most recent simulation-kernel launch
+    bool ev_valid;
 };
 
 extern thread_local char g_last_cuda_error[256];
