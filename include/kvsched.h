@@ -161,6 +161,27 @@ int sched_local_search(sched_handle h, int neighbourhood, int32_t iters, uint64_
  * that launch.  Waits for the launch to finish.  SCHED_E_INVAL if there was none. */
 int sched_last_eval_kernel_ms(sched_handle h, float* ms_out);
 
+/* Arg-min over a TEL array without any allocation (the paper has no counterpart; this exists for
+ * callers that are not allowed to allocate device memory: a serving process whose memory pool
+ * already owns the whole GPU, a plug-in that works inside buffers it was given, a latency-critical
+ * loop that must stay clear of the allocator's device-wide synchronisation).  No handle is needed.
+ *   tel        : device int64[count], e.g. the tel_out of sched_sweep_dev.
+ *   count      : 1 .. 2^26 candidates; larger counts are refused with SCHED_E_UNSUPPORTED (and a
+ *                message in sched_last_cuda_error()), smaller or NULL arguments with SCHED_E_INVAL.
+ *   index_base : added to the position of the winner (first move code / sample index of `tel`).
+ *   best_out   : device int64[2] = {min TEL, lowest index attaining it}; same result as the
+ *                best_out of sched_sweep_dev on the same TELs.
+ *   cuda_stream: cudaStream_t (as void*) to enqueue on, NULL for the default stream; asynchronous.
+ * Works on the CUDA device that is current in the calling thread.  Its partial results and ticket
+ * counter live in a 16.25 KiB array inside the library image, present on every GPU that loads the
+ * library until the process exits; this call never calls cudaMalloc/cudaFree or any allocating
+ * routine.  The first call on each device looks up that array's device address (make that first
+ * call before starting any stream capture).  All calls on a device share the array and it keeps the
+ * previous call's contents (the counter is cleared on the stream before each launch), so two calls
+ * whose kernels may overlap on one GPU race: order them on one stream or with events. */
+int sched_argmin_static_dev(const int64_t* tel, int64_t count, int64_t index_base,
+                            int64_t* best_out, void* cuda_stream);
+
 /* Counters since sched_init: kernels launched by this handle, candidates evaluated. */
 int sched_stats(sched_handle h, int64_t* kernel_launches_out, int64_t* evaluations_out);
 

@@ -22,7 +22,7 @@ NBHD_SWAP, NBHD_SWAP_INSERT, NBHD_SAMPLED = 0, 1, 2
 EXPORTS = [
     "sched_init", "sched_init_batch", "sched_set_stream", "sched_sync", "sched_set_base_order",
     "sched_get_base_order", "sched_eval_batch", "sched_eval_batch_dev", "sched_sweep_dev",
-    "sched_sorted_f", "sched_sorted_f_dev", "sched_local_search", "sched_last_eval_kernel_ms", "sched_stats", "sched_destroy",
+    "sched_sorted_f", "sched_sorted_f_dev", "sched_local_search", "sched_last_eval_kernel_ms", "sched_argmin_static_dev", "sched_stats", "sched_destroy",
     "sched_strerror", "sched_last_cuda_error",
 ]
 
@@ -66,6 +66,7 @@ def load():
     lib.sched_local_search.argtypes = [vp, C.c_int, i32, u64, i64, vp, vp, vp, vp]
     lib.sched_stats.argtypes = [vp, vp, vp]
     lib.sched_last_eval_kernel_ms.argtypes = [vp, vp]
+    lib.sched_argmin_static_dev.argtypes = [vp, i64, i64, vp, vp]
     lib.sched_destroy.argtypes = [vp]
     lib.sched_strerror.argtypes = [C.c_int]
     lib.sched_strerror.restype = C.c_char_p
@@ -226,3 +227,15 @@ class Scheduler:
                                          C.byref(tel), C.byref(done), _np_ptr(trace)), "sched_local_search")
         final = buf if buf is not None else self.get_base_order()
         return final, tel.value, done.value, trace[:done.value].copy()
+
+
+def argmin_static_dev(tel, best_out, *, count=None, index_base=0, stream=None):
+    """Best (TEL, index) of a device TEL tensor through ``sched_argmin_static_dev``: the variant of
+    the arg-min that allocates nothing, for callers that may not touch the device allocator (its
+    scratch is a fixed array inside the library).  ``tel``/``best_out`` are CUDA int64 tensors on the
+    current device; asynchronous on ``stream`` (a torch.cuda.Stream) or the default stream.  Calls
+    that could overlap on one GPU must be ordered by the caller: they share the scratch array."""
+    n = int(tel.numel()) if count is None else int(count)
+    ptr = C.c_void_p(stream.cuda_stream) if stream is not None else None
+    _check(load().sched_argmin_static_dev(_dev_ptr(tel), n, index_base, _dev_ptr(best_out), ptr),
+           "sched_argmin_static_dev")

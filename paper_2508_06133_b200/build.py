@@ -1,4 +1,4 @@
-"""Builds the CUDA library in-tree: ``csrc/api.cu`` -> ``libkvsched.so`` (sm_100a only)."""
+"""Builds the CUDA library in-tree: ``csrc/*.cu`` -> ``libkvsched.so`` (sm_100a only)."""
 from __future__ import annotations
 
 import os
@@ -27,7 +27,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if force or stale():
         nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
         tmp = LIB + ".%d.tmp" % os.getpid()
-        cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + [os.path.join(CSRC, "api.cu"), "-o", tmp]
+        cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + [os.path.join(CSRC, "api.cu"), os.path.join(CSRC, "argmin_static.cu"), "-o", tmp]
         subprocess.check_call(cmd)
         os.replace(tmp, LIB)
     return LIB
