@@ -26,6 +26,17 @@ namespace {
 const i64 kSweepChunk = 1ll << 22;          // candidates per launch inside a sweep
 const size_t kSnapBudget = 512ull << 20;    // bytes of snapshot memory before striding kicks in
 
+// Runs `call(NIT)` for the handle's simulator shape.
+#define KV_DISPATCH_NIT(nit, CALL)            \
+    switch (nit) {                             \
+        case 1: CALL(1); break;                \
+        case 2: CALL(2); break;                \
+        case 3: CALL(3); break;                \
+        case 5: CALL(5); break;                \
+        case 9: CALL(9); break;                \
+        default: CALL(0); break;               \
+    }
+
 int bits_of(u64 v) { int b = 0; while (v) { ++b; v >>= 1; } return b; }
 
 // byte mask for a 64-bit key whose low word uses lo_bits and high word hi_bits
@@ -141,6 +152,7 @@ int create_common(sched_ctx** out, int B, int n, const int32_t* s, const int32_t
         h->smem_optin = (int)prop.sharedMemPerBlockOptin;
         h->B = B; h->n = n; h->M = M; h->omax = omax; h->sum_o_max = sum_max;
         h->L = (omax + 8 + 3) & ~3;
+        h->nit = sim_pick_nit(omax);
         if ((size_t)K3_WARPS * h->L * sizeof(int) > (size_t)h->smem_optin - 2048) { rc = SCHED_E_UNSUPPORTED; break; }
         if (cudaStreamCreateWithFlags(&h->own_stream, cudaStreamNonBlocking) != cudaSuccess) { rc = kv_cuda_fail(cudaGetLastError(), "cudaStreamCreate"); break; }
         h->stream = h->own_stream;
@@ -186,11 +198,21 @@ int create_common(sched_ctx** out, int B, int n, const int32_t* s, const int32_t
             C(cudaMemcpyAsync(h->d_seg_off, seg, sizeof(seg), cudaMemcpyHostToDevice, st));
         }
         // opt in to large dynamic shared memory once
-        C(cudaFuncSetAttribute(k3_eval_moves, cudaFuncAttributeMaxDynamicSharedMemorySize, h->smem_optin - 2048));
-        C(cudaFuncSetAttribute(k3_eval_orders, cudaFuncAttributeMaxDynamicSharedMemorySize, h->smem_optin - 2048));
+        {
+            const int dyn = h->smem_optin - 2048;
+            cudaError_t e1 = cudaSuccess, e2 = cudaSuccess, e3 = cudaSuccess, e4 = cudaSuccess;
+#define SETATTR(N)                                                                                         \
+            e1 = cudaFuncSetAttribute(k3_eval_moves<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn);  \
+            e2 = cudaFuncSetAttribute(k3_eval_orders<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn); \
+            e3 = cudaFuncSetAttribute(k3_eval_policy<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn); \
+            e4 = cudaFuncSetAttribute(k3_base_run<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn)
+            KV_DISPATCH_NIT(h->nit, SETATTR);
+#undef SETATTR
+            if (e1 != cudaSuccess || e2 != cudaSuccess || e3 != cudaSuccess || e4 != cudaSuccess) {
+                rc = kv_cuda_fail(cudaGetLastError(), "cudaFuncSetAttribute(MaxDynamicSharedMemorySize)"); break;
+            }
+        }
         C(cudaFuncSetAttribute(k3_check_starts, cudaFuncAttributeMaxDynamicSharedMemorySize, h->smem_optin - 2048));
-        C(cudaFuncSetAttribute(k3_eval_policy, cudaFuncAttributeMaxDynamicSharedMemorySize, h->smem_optin - 2048));
-        C(cudaFuncSetAttribute(k3_base_run, cudaFuncAttributeMaxDynamicSharedMemorySize, h->smem_optin - 2048));
         C(cudaStreamSynchronize(st));       // s, o may be pageable host memory owned by the caller
 #undef C
     } while (0);
@@ -205,9 +227,11 @@ int ensure_base(sched_ctx* h) {
     const int n = h->n;
     k3_gather_table<<<(n + 255) / 256, 256, 0, h->stream>>>(h->d_tbl_id, h->d_order, n, h->d_tbl_base);
     KV_TRY(check_launch(h));
-    k3_base_run<<<1, 32, (size_t)h->L * sizeof(int), h->stream>>>(
-        h->d_tbl_base, n, h->L, (int)h->M, h->snap_stride, h->d_snap_ring, h->d_snap_hdr,
-        h->d_base_starts, h->d_base_tel, h->d_status);
+#define RUN(N) k3_base_run<N><<<1, 32, (size_t)h->L * sizeof(int), h->stream>>>(                    \
+        h->d_tbl_base, n, h->L, (int)h->M, h->snap_stride, h->d_snap_ring, h->d_snap_hdr,            \
+        h->d_base_starts, h->d_base_tel, h->d_status)
+    KV_DISPATCH_NIT(h->nit, RUN);
+#undef RUN
     KV_TRY(check_launch(h));
     h->base_ready = true;
     return SCHED_OK;
@@ -238,7 +262,9 @@ int launch_moves(sched_ctx* h, int mode, const i64* codes, i64 first, u64 seed, 
     p.counter = h->d_counter; p.status = h->d_status;
     KV_CUDA(cudaMemsetAsync(h->d_counter, 0, sizeof(unsigned), h->stream));
     KV_CUDA(cudaEventRecord(h->ev_k3_begin, h->stream));
-    k3_eval_moves<<<k3_grid(h, count), K3_THREADS, smem, h->stream>>>(p);
+#define RUN(N) k3_eval_moves<N><<<k3_grid(h, count), K3_THREADS, smem, h->stream>>>(p)
+    KV_DISPATCH_NIT(h->nit, RUN);
+#undef RUN
     KV_TRY(check_launch(h));
     KV_CUDA(cudaEventRecord(h->ev_k3_end, h->stream));
     h->ev_valid = true;
@@ -339,9 +365,11 @@ int sched_eval_batch_dev(sched_handle h, int kind, int64_t count, const void* ca
         if (smem > (size_t)h->smem_optin - 2048) return SCHED_E_UNSUPPORTED;
         const i64 ctas = (i64)h->B * count;
         if (ctas >= (1ll << 31)) return SCHED_E_UNSUPPORTED;
-        k3_eval_policy<<<(unsigned)ctas, 32, smem, h->stream>>>(h->d_s, h->d_o, n, h->L, (int)h->M,
-                                                                  (const int*)candidates, (int)count,
-                                                                  (i64*)tel_out, starts_out, h->d_status);
+#define RUN(N) k3_eval_policy<N><<<(unsigned)ctas, 32, smem, h->stream>>>(h->d_s, h->d_o, n, h->L, (int)h->M, \
+                                                                  (const int*)candidates, (int)count,        \
+                                                                  (i64*)tel_out, starts_out, h->d_status)
+        KV_DISPATCH_NIT(h->nit, RUN);
+#undef RUN
         KV_TRY(check_launch(h));
         h->evaluations += ctas;
         if (feasible_out) KV_CUDA(cudaMemsetAsync(feasible_out, 1, (size_t)ctas, h->stream));
@@ -364,7 +392,9 @@ int sched_eval_batch_dev(sched_handle h, int kind, int64_t count, const void* ca
         p.counter = h->d_counter; p.status = h->d_status;
         KV_CUDA(cudaMemsetAsync(h->d_counter, 0, sizeof(unsigned), h->stream));
         KV_CUDA(cudaEventRecord(h->ev_k3_begin, h->stream));
-        k3_eval_orders<<<k3_grid(h, count), K3_THREADS, smem, h->stream>>>(p);
+#define RUN(N) k3_eval_orders<N><<<k3_grid(h, count), K3_THREADS, smem, h->stream>>>(p)
+        KV_DISPATCH_NIT(h->nit, RUN);
+#undef RUN
         KV_TRY(check_launch(h));
         KV_CUDA(cudaEventRecord(h->ev_k3_end, h->stream));
         h->ev_valid = true;

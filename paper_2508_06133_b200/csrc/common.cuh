@@ -29,6 +29,7 @@ struct sched_ctx {
     i64 M;
     int omax;                // largest decode length over all instances
     int L;                   // ring length in cells (multiple of 4, >= omax + 8)
+    int nit;                 // simulator shape: 128-cell rounds cached in registers (0: streamed)
     i64 sum_o_max;           // largest sum of o over instances (bounds every start time)
     int sm_count;
     int smem_optin;          // max dynamic shared memory per block (bytes)

@@ -94,6 +94,7 @@ __global__ void k3_iota(int* a, int n) {
 // Base run: positions 0 .. n-1 of the base order; snapshot idx holds the state in front of
 // position idx * stride.  One warp.  Dynamic shared memory: L ints.
 // ------------------------------------------------------------------------------------------------
+template <int NIT>
 __global__ void __launch_bounds__(32)
 k3_base_run(const int2* __restrict__ tbl_base, int n, int L, int M, int stride,
             int* __restrict__ snap_ring, SnapHeader* __restrict__ snap_hdr,
@@ -119,7 +120,7 @@ k3_base_run(const int2* __restrict__ tbl_base, int n, int L, int M, int stride,
                 }
             }
             const int s = __shfl_sync(KV_FULL, so.x, k), o = __shfl_sync(KV_FULL, so.y, k);
-            const int p = sim_admit(ring, L, M, st, s, o, lane, status);
+            const int p = sim_admit<NIT>(ring, L, M, st, s, o, lane, status);
             if (lane == 0) base_starts_pos[q] = p;
         }
     }
@@ -150,6 +151,7 @@ struct MoveEvalParams {
     int* status;
 };
 
+template <int NIT>
 __global__ void __launch_bounds__(K3_THREADS, 1)
 k3_eval_moves(const MoveEvalParams p) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -201,7 +203,7 @@ k3_eval_moves(const MoveEvalParams p) {
             const int cnt = min(32, n - q0);
             for (int k = 0; k < cnt; ++k) {
                 const int s = __shfl_sync(KV_FULL, so.x, k), o = __shfl_sync(KV_FULL, so.y, k);
-                const int pstart = sim_admit(ring, L, M, st, s, o, lane, p.status);
+                const int pstart = sim_admit<NIT>(ring, L, M, st, s, o, lane, p.status);
                 if (starts && lane == k) starts[id] = pstart;
             }
         }
@@ -225,6 +227,7 @@ struct OrderEvalParams {
     int* status;
 };
 
+template <int NIT>
 __global__ void __launch_bounds__(K3_THREADS, 1)
 k3_eval_orders(const OrderEvalParams p) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -257,7 +260,7 @@ k3_eval_orders(const OrderEvalParams p) {
             const int cnt = min(32, n - q0);
             for (int k = 0; k < cnt; ++k) {
                 const int s = __shfl_sync(KV_FULL, so.x, k), o = __shfl_sync(KV_FULL, so.y, k);
-                const int pstart = sim_admit(ring, L, M, st, s, o, lane, p.status);
+                const int pstart = sim_admit<NIT>(ring, L, M, st, s, o, lane, p.status);
                 if (starts && lane == k) starts[id] = pstart;
             }
         }
@@ -267,8 +270,8 @@ k3_eval_orders(const OrderEvalParams p) {
 
 // ------------------------------------------------------------------------------------------------
 // Policy sweep: grid = B * P single-warp CTAs; CTA (b, k) evaluates instance b under policies[k].
-// Dynamic shared memory: int s[n], o[n], ord[n], tmp[n]; u64 key[n]; i64 P[n+1], O[n+1]; int boff[n+1];
-// int ring[L].
+// Dynamic shared memory: int ring[L]; i64 P[n+1], O[n+1]; u64 key[n]; int s[n], o[n], ord[n], tmp[n],
+// boff[n+2].
 // ------------------------------------------------------------------------------------------------
 __device__ __forceinline__ void k3_rank_sort(const u64* key, const int* ids_in, int* ids_out, int lo, int hi, int lane) {
     // ids_out[lo + rank] = ids_in[e]; rank by (key, position) -- keys carry their own tie-breakers
@@ -284,6 +287,7 @@ __device__ __forceinline__ void k3_rank_sort(const u64* key, const int* ids_in, 
     __syncwarp();
 }
 
+template <int NIT>
 __global__ void __launch_bounds__(32)
 k3_eval_policy(const int* __restrict__ s_all, const int* __restrict__ o_all, int n, int L, int M,
                const int* __restrict__ policies, int num_policies,
@@ -292,7 +296,8 @@ k3_eval_policy(const int* __restrict__ s_all, const int* __restrict__ o_all, int
     const int lane = threadIdx.x;
     const int b = blockIdx.x / num_policies, kpol = blockIdx.x % num_policies;
     const int policy = policies[kpol];
-    i64* P = (i64*)smem_raw;
+    int* ring = (int*)smem_raw;                       // first: 16-byte aligned for the vector loads
+    i64* P = (i64*)(ring + L);                        // L is a multiple of 4
     i64* O = P + (n + 1);
     u64* key = (u64*)(O + (n + 1));
     int* s = (int*)(key + n);
@@ -300,7 +305,6 @@ k3_eval_policy(const int* __restrict__ s_all, const int* __restrict__ o_all, int
     int* ord = o + n;
     int* tmp = ord + n;
     int* boff = tmp + n;
-    int* ring = boff + (n + 2);
     __shared__ i64 sh_warp[64];
     __shared__ i64 carry[2];
     __shared__ u64 sh_best[66];
@@ -342,7 +346,7 @@ k3_eval_policy(const int* __restrict__ s_all, const int* __restrict__ o_all, int
     int* starts = starts_out ? starts_out + ((size_t)b * num_policies + kpol) * n : nullptr;
     for (int q = 0; q < n; ++q) {
         const int id = ord[q];
-        const int pstart = sim_admit(ring, L, M, st, s[id], o[id], lane, status);
+        const int pstart = sim_admit<NIT>(ring, L, M, st, s[id], o[id], lane, status);
         if (starts && lane == 0) starts[id] = pstart;
     }
     if (lane == 0) tel_out[(size_t)b * num_policies + kpol] = st.tel;

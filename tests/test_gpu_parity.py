@@ -78,6 +78,27 @@ def test_orders_long_waits_and_ring_wrap():
             assert tel[c] == t and (starts[c] == p).all()
 
 
+@pytest.mark.parametrize("omax", [100, 122, 123, 250, 251, 378, 379, 634, 635, 1100, 1146, 1147, 1500, 3000])
+def test_orders_every_simulator_shape(omax):
+    """Window lengths around each register-cached shape's limit, and the streamed shape beyond."""
+    rng = np.random.default_rng(omax)
+    n, M = 90, 4 * omax
+    s = rng.integers(1, omax, n).astype(np.int32)
+    o = rng.integers(1, omax + 1, n).astype(np.int32)
+    o[:6] = [omax, omax - 1, 1, 2, 3, omax]
+    s[::11] = M - o[::11]
+    orders = np.stack([rng.permutation(n) for _ in range(4)]).astype(np.int32)
+    with kv.Scheduler(s, o, M) as h:
+        tel, _, starts = h.eval_batch(kv.CAND_ORDER, orders, want_starts=True)
+        h.set_base_order(orders[0])
+        codes = all_codes(n)[::37]
+        mtel, _, _ = h.eval_batch(kv.CAND_MOVE, codes)
+    for c in range(4):
+        p, tt, _ = orc.list_schedule_rounds(s, o, M, orders[c])
+        assert tel[c] == tt and (starts[c] == p).all()
+    assert (mtel == oracle_moves(s, o, M, orders[0], codes)).all()
+
+
 def test_orders_mixed_1k():
     inst = W.mixed_1k()
     orders = W.random_permutations(inst.n, 6, seed=9)
