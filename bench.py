@@ -244,7 +244,7 @@ def main():
     roof_smem = {"bound": "smem", "achieved": smem_ach, "peak": smem_peak, "unit": "GB/s", "frac": smem_ach / smem_peak}
     roof_alu = {"bound": "alu", "achieved": alu_ach, "peak": alu_peak, "unit": "Tint-op/s", "frac": alu_ach / alu_peak}
     roofline = dict(roof_alu)
-    ring_cells = (int(inst.o.max()) + 8 + 3) & ~3
+    ring_cells = (int(inst.o.max()) + 8 + 31) & ~31
     hbm_bytes = 4.0 * n * ring_cells + 8.0 * count + 8.0 * n      # snapshots read once, TELs out, request table
     roofline.update({"traffic": None, "kernel": "k3_eval_moves", "kernel_ms": kern_s * 1e3,
                      "cells_per_launch": cells_per_launch,

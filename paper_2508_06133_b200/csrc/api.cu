@@ -31,9 +31,8 @@ const size_t kSnapBudget = 512ull << 20;    // bytes of snapshot memory before s
     switch (nit) {                             \
         case 1: CALL(1); break;                \
         case 2: CALL(2); break;                \
-        case 3: CALL(3); break;                \
-        case 5: CALL(5); break;                \
-        case 9: CALL(9); break;                \
+        case 4: CALL(4); break;                \
+        case 8: CALL(8); break;                \
         default: CALL(0); break;               \
     }
 
@@ -151,7 +150,7 @@ int create_common(sched_ctx** out, int B, int n, const int32_t* s, const int32_t
         h->sm_count = prop.multiProcessorCount;
         h->smem_optin = (int)prop.sharedMemPerBlockOptin;
         h->B = B; h->n = n; h->M = M; h->omax = omax; h->sum_o_max = sum_max;
-        h->L = (omax + 8 + 3) & ~3;
+        h->L = (omax + 8 + 31) & ~31;          // multiple of 32 cells: a wrapped 16-byte access keeps its bank
         h->nit = sim_pick_nit(omax);
         if ((size_t)K3_WARPS * h->L * sizeof(int) > (size_t)h->smem_optin - 2048) { rc = SCHED_E_UNSUPPORTED; break; }
         if (cudaStreamCreateWithFlags(&h->own_stream, cudaStreamNonBlocking) != cudaSuccess) { rc = kv_cuda_fail(cudaGetLastError(), "cudaStreamCreate"); break; }

@@ -28,7 +28,7 @@ struct sched_ctx {
     int B, n;                // instances, requests per instance
     i64 M;
     int omax;                // largest decode length over all instances
-    int L;                   // ring length in cells (multiple of 4, >= omax + 8)
+    int L;                   // ring length in cells (multiple of 32, >= omax + 8)
     int nit;                 // simulator shape: 128-cell rounds cached in registers (0: streamed)
     i64 sum_o_max;           // largest sum of o over instances (bounds every start time)
     int sm_count;

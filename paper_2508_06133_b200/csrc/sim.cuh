@@ -26,7 +26,7 @@
 // stay fine when p grows, so only the cells that enter the window on the right are looked at again.
 //
 // Two code shapes with identical results:
-//   sim_admit<NIT>, NIT >= 1: the window (<= 128*NIT - 6 cells) is loaded once with 16-byte shared
+//   sim_admit<NIT>, NIT >= 1: the window (<= 128*NIT + 3 cells) is loaded once with 16-byte shared
 //     loads into registers, checked, and written back -- one read and one write per cell;
 //   sim_admit<0>: any window length, cells are re-read by the write pass.
 #pragma once
@@ -92,83 +92,97 @@ __device__ __forceinline__ void sim_finish_beyond(int* __restrict__ ring, int L,
 }
 
 // Admit one request; returns its start time.  All 32 lanes call this with identical arguments.
+//
+// Register-cached form: the window [t, t+o) is split at 16-byte boundaries of the ring into a head
+// (0..3 cells, lanes 0..2), a body of full 4-cell groups (group g of round `it` belongs to lane
+// g - 32*it; no masks needed) and a tail (0..3 cells, lanes 4..6).
 template <int NIT>
 __device__ __forceinline__ int sim_admit(int* __restrict__ ring, int L, int M, SimState& st,
                                          int s, int o, int lane, int* status) {
     const int t = st.t, tr = st.tr;
-    const int m = tr & 3, ar = tr - m;               // L is a multiple of 4: t and tr agree mod 4
-    const int span = m + o;                          // cells from the aligned start to the window end
-    const int nit = (span + 127) >> 7;               // 16-byte groups: 32 lanes x 4 cells per round
     const int kadm = s + 1 - M - t;                  // V + kadm > 0  <=>  the cell is over budget
     const int kw = s + 1;                            // ramp value at the window start
-    const int g4l = lane << 2;
     int delta = 0;
 
     if (NIT > 0) {
+        const int h = (4 - (tr & 3)) & 3;            // L is a multiple of 4: t and tr agree mod 4
+        const int hc = o < h ? o : h;                // head cells
+        const int nbody = (o - hc) >> 2;             // full groups
+        const int tc = (o - hc) & 3;                 // tail cells
+        const int nit = (nbody + 31) >> 5;
+        const int ab = kv_wrap1(tr + hc, L);         // ring index of the first body cell (16-byte aligned)
+        // scalar cell of this lane: head cell `lane` or tail cell `lane - 4`
+        int sr = -1;
+        if (lane < hc) sr = lane;
+        else if ((unsigned)(lane - 4) < (unsigned)tc) sr = hc + (nbody << 2) + lane - 4;
+        int sidx = 0, sv = -1;
+        if (sr >= 0) { sidx = kv_wrap1(tr + sr, L); sv = ring[sidx]; }
         int4 buf[NIT > 0 ? NIT : 1];
-        int vmax = -1;
+        int vmax = sv;
 #pragma unroll
         for (int it = 0; it < NIT; ++it) {
             if (it >= nit) break;
-            const int g4 = g4l + (it << 7);
+            const int g = lane + (it << 5);
             int4 v = make_int4(-1, -1, -1, -1);
-            if (g4 < span) v = *reinterpret_cast<const int4*>(ring + kv_wrap1(ar + g4, L));
+            if (g < nbody) v = *reinterpret_cast<const int4*>(ring + kv_wrap1(ab + (g << 2), L));
             buf[it] = v;
-            const int lim = span - g4;               // cells c >= lim are past the window end
-            const int mm = it == 0 ? m - g4 : 0;     // cells c < mm are before the window start
-            if (it == 0) { if (0 < mm) v.x = -1; if (1 < mm) v.y = -1; if (2 < mm) v.z = -1; }
-            if (it == nit - 1) { if (lim < 4) { v.w = -1; if (lim < 3) v.z = -1; if (lim < 2) v.y = -1; if (lim < 1) v.x = -1; } }
             vmax = max(max(vmax, max(v.x, v.y)), max(v.z, v.w));
         }
         vmax = kv_warp_max(vmax);
-        if (vmax + kadm > 0) {
-            // blocked: advance implied by the cells of the window
-            int need = 0;
+        const int rl = hc + (lane << 2);             // window offset of this lane's group in round 0
+        if (vmax + kadm <= 0) {
+            if (sr >= 0) ring[sidx] = sv + kw + sr;
 #pragma unroll
             for (int it = 0; it < NIT; ++it) {
                 if (it >= nit) break;
-                const int r0 = g4l + (it << 7) - m;
+                const int g = lane + (it << 5);
+                if (g < nbody) {
+                    int4 v = buf[it];
+                    const int k0 = kw + rl + (it << 7);
+                    v.x += k0; v.y += k0 + 1; v.z += k0 + 2; v.w += k0 + 3;
+                    *reinterpret_cast<int4*>(ring + kv_wrap1(ab + (g << 2), L)) = v;
+                }
+            }
+        } else {
+            // blocked: advance implied by the cells of the window (empty filler cells hold -1)
+            int need = 0;
+            if (sr >= 0) need = min(sv + kadm, sr + 1);
+#pragma unroll
+            for (int it = 0; it < NIT; ++it) {
+                if (it >= nit) break;
                 const int4 v = buf[it];
-                if ((unsigned)(r0 + 0) < (unsigned)o) need = max(need, min(v.x + kadm, r0 + 1));
-                if ((unsigned)(r0 + 1) < (unsigned)o) need = max(need, min(v.y + kadm, r0 + 2));
-                if ((unsigned)(r0 + 2) < (unsigned)o) need = max(need, min(v.z + kadm, r0 + 3));
-                if ((unsigned)(r0 + 3) < (unsigned)o) need = max(need, min(v.w + kadm, r0 + 4));
+                if (max(max(v.x, v.y), max(v.z, v.w)) + kadm > 0) {
+                    const int r1 = rl + (it << 7) + 1;
+                    need = max(need, max(max(min(v.x + kadm, r1), min(v.y + kadm, r1 + 1)),
+                                         max(min(v.z + kadm, r1 + 2), min(v.w + kadm, r1 + 3))));
+                }
             }
             delta = kv_warp_max(need);
-            delta = sim_search_beyond(ring, L, t, tr, st.hz - t, o, kadm, delta, lane, status);
+            const int live = st.hz - t;
+            if (o < live) delta = sim_search_beyond(ring, L, t, tr, live, o, kadm, delta, lane, status);
             const int kwd = kw - delta, dead = t + L;
+            if (sr >= 0) ring[sidx] = sr >= delta ? sv + kwd + sr : dead + sr;
 #pragma unroll
             for (int it = 0; it < NIT; ++it) {
                 if (it >= nit) break;
-                const int g4 = g4l + (it << 7), r0 = g4 - m;
-                if (g4 < span) {
+                const int g = lane + (it << 5);
+                if (g < nbody) {
                     int4 v = buf[it];
-                    if ((unsigned)(r0 + 0) < (unsigned)o) v.x = r0 + 0 >= delta ? v.x + kwd + r0 + 0 : dead + r0 + 0;
-                    if ((unsigned)(r0 + 1) < (unsigned)o) v.y = r0 + 1 >= delta ? v.y + kwd + r0 + 1 : dead + r0 + 1;
-                    if ((unsigned)(r0 + 2) < (unsigned)o) v.z = r0 + 2 >= delta ? v.z + kwd + r0 + 2 : dead + r0 + 2;
-                    if ((unsigned)(r0 + 3) < (unsigned)o) v.w = r0 + 3 >= delta ? v.w + kwd + r0 + 3 : dead + r0 + 3;
-                    *reinterpret_cast<int4*>(ring + kv_wrap1(ar + g4, L)) = v;
+                    const int r0 = rl + (it << 7);
+                    if (r0 >= delta) {
+                        const int k0 = kwd + r0;
+                        v.x += k0; v.y += k0 + 1; v.z += k0 + 2; v.w += k0 + 3;
+                    } else {
+                        v.x = dead + r0;                                              // r0 < delta
+                        v.y = r0 + 1 >= delta ? v.y + kwd + r0 + 1 : dead + r0 + 1;
+                        v.z = r0 + 2 >= delta ? v.z + kwd + r0 + 2 : dead + r0 + 2;
+                        v.w = r0 + 3 >= delta ? v.w + kwd + r0 + 3 : dead + r0 + 3;
+                    }
+                    *reinterpret_cast<int4*>(ring + kv_wrap1(ab + (g << 2), L)) = v;
                 }
             }
             __syncwarp();
             sim_finish_beyond(ring, L, t, tr, o, kw, delta, lane);
-        } else {
-#pragma unroll
-            for (int it = 0; it < NIT; ++it) {
-                if (it >= nit) break;
-                const int g4 = g4l + (it << 7);
-                if (g4 < span) {
-                    int4 v = buf[it];
-                    const int lim = span - g4;
-                    const int mm = it == 0 ? m - g4 : 0;
-                    const int kr = kw + g4 - m;      // ramp value of this group's first cell
-                    int ax = kr, ay = kr + 1, az = kr + 2, aw = kr + 3;
-                    if (it == 0) { if (0 < mm) ax = 0; if (1 < mm) ay = 0; if (2 < mm) az = 0; }
-                    if (it == nit - 1) { if (lim < 4) { aw = 0; if (lim < 3) az = 0; if (lim < 2) ay = 0; } }
-                    v.x += ax; v.y += ay; v.z += az; v.w += aw;
-                    *reinterpret_cast<int4*>(ring + kv_wrap1(ar + g4, L)) = v;
-                }
-            }
         }
     } else {
         // streamed form: same arithmetic, cells re-read instead of cached
@@ -201,8 +215,8 @@ __device__ __forceinline__ int sim_admit(int* __restrict__ ring, int L, int M, S
 
 // Number of 128-cell rounds a handle's longest window needs (0: use the streamed form).
 static inline int sim_pick_nit(int omax) {
-    const int need = (omax + 3 + 127) / 128;          // span <= 3 + omax
-    const int sizes[] = {1, 2, 3, 5, 9};
-    for (int k = 0; k < 5; ++k) if (need <= sizes[k]) return sizes[k];
+    const int need = (omax / 4 + 31) / 32;            // full 4-cell groups of the longest window
+    const int sizes[] = {1, 2, 4, 8};
+    for (int k = 0; k < 4; ++k) if (need <= sizes[k]) return sizes[k];
     return 0;
 }

@@ -78,7 +78,7 @@ def test_orders_long_waits_and_ring_wrap():
             assert tel[c] == t and (starts[c] == p).all()
 
 
-@pytest.mark.parametrize("omax", [100, 122, 123, 250, 251, 378, 379, 634, 635, 1100, 1146, 1147, 1500, 3000])
+@pytest.mark.parametrize("omax", [100, 127, 128, 129, 255, 256, 257, 511, 512, 513, 1023, 1024, 1025, 1500, 3000])
 def test_orders_every_simulator_shape(omax):
     """Window lengths around each register-cached shape's limit, and the streamed shape beyond."""
     rng = np.random.default_rng(omax)
