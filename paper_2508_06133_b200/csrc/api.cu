@@ -26,14 +26,26 @@ namespace {
 const i64 kSweepChunk = 1ll << 22;          // candidates per launch inside a sweep
 const size_t kSnapBudget = 512ull << 20;    // bytes of snapshot memory before striding kicks in
 
-// Runs `call(NIT)` for the handle's simulator shape.
-#define KV_DISPATCH_NIT(nit, CALL)            \
-    switch (nit) {                             \
-        case 1: CALL(1); break;                \
-        case 2: CALL(2); break;                \
-        case 4: CALL(4); break;                \
-        case 8: CALL(8); break;                \
-        default: CALL(0); break;               \
+// Runs CALL(SIM) with SIM = the simulator class of the handle: the register-resident one when the
+// longest window fits 33 registers per lane, else the shared-memory one.
+#define KV_DISPATCH_SIM(h, CALL)                               \
+    if ((h)->nreg > 0) {                                        \
+        switch ((h)->nreg) {                                    \
+            case 2: CALL(RegSim<2>); break;                     \
+            case 3: CALL(RegSim<3>); break;                     \
+            case 5: CALL(RegSim<5>); break;                     \
+            case 9: CALL(RegSim<9>); break;                     \
+            case 17: CALL(RegSim<17>); break;                   \
+            default: CALL(RegSim<33>); break;                   \
+        }                                                       \
+    } else {                                                    \
+        switch ((h)->nit) {                                     \
+            case 1: CALL(SmemSim<1>); break;                    \
+            case 2: CALL(SmemSim<2>); break;                    \
+            case 4: CALL(SmemSim<4>); break;                    \
+            case 8: CALL(SmemSim<8>); break;                    \
+            default: CALL(SmemSim<0>); break;                   \
+        }                                                       \
     }
 
 int bits_of(u64 v) { int b = 0; while (v) { ++b; v >>= 1; } return b; }
@@ -114,8 +126,20 @@ void free_ctx(sched_ctx* h) {
     delete h;
 }
 
+int k3_warps(const sched_ctx* h) {
+    int w = 0;
+#define GETW(SIM) w = SIM::kWarps
+    KV_DISPATCH_SIM(h, GETW);
+#undef GETW
+    if (h->nreg == 0) {                       // one ring per warp has to fit in shared memory
+        const int fit = (int)(((size_t)h->smem_optin - 2048) / ((size_t)h->L * sizeof(int)));
+        if (fit < w) w = fit;
+    }
+    return w;
+}
+
 size_t k3_smem_bytes(const sched_ctx* h, bool* table_in_smem, unsigned* table_bytes) {
-    const size_t rings = (size_t)K3_WARPS * h->L * sizeof(int);
+    const size_t rings = h->nreg > 0 ? 0 : (size_t)k3_warps(h) * h->L * sizeof(int);
     const unsigned tb = (unsigned)(((size_t)h->n * sizeof(int2) + 15) & ~(size_t)15);
     const size_t with_table = ((size_t)tb + 127) / 128 * 128 + rings;
     if (with_table <= (size_t)h->smem_optin - 2048) {
@@ -150,9 +174,18 @@ int create_common(sched_ctx** out, int B, int n, const int32_t* s, const int32_t
         h->sm_count = prop.multiProcessorCount;
         h->smem_optin = (int)prop.sharedMemPerBlockOptin;
         h->B = B; h->n = n; h->M = M; h->omax = omax; h->sum_o_max = sum_max;
-        h->L = (omax + 8 + 31) & ~31;          // multiple of 32 cells: a wrapped 16-byte access keeps its bank
+        h->nreg = sim_pick_nreg(omax);
+        if (const char* kind = getenv("KVSCHED_SIM"))               // testing knob: "smem" forces the shared-memory simulator
+            if (strcmp(kind, "smem") == 0) h->nreg = 0;
         h->nit = sim_pick_nit(omax);
-        if ((size_t)K3_WARPS * h->L * sizeof(int) > (size_t)h->smem_optin - 2048) { rc = SCHED_E_UNSUPPORTED; break; }
+        if (const char* cap = getenv("KVSCHED_MAX_NIT")) {          // tuning knob: windows beyond the cap stream
+            const int c = atoi(cap);
+            if (c == 0 || c == 1 || c == 2 || c == 4 || c == 8) h->nit = c < h->nit ? c : h->nit;
+        }
+        // cells per simulator state: registers x 32 lanes, or a ring whose length is a multiple of
+        // 32 cells (a wrapped 16-byte access then keeps its bank)
+        h->L = h->nreg > 0 ? 32 * h->nreg : (omax + 8 + 31) & ~31;
+        if (k3_warps(h) < 1) { rc = SCHED_E_UNSUPPORTED; break; }
         if (cudaStreamCreateWithFlags(&h->own_stream, cudaStreamNonBlocking) != cudaSuccess) { rc = kv_cuda_fail(cudaGetLastError(), "cudaStreamCreate"); break; }
         h->stream = h->own_stream;
         if (cudaEventCreate(&h->ev_k3_begin) != cudaSuccess || cudaEventCreate(&h->ev_k3_end) != cudaSuccess) { rc = kv_cuda_fail(cudaGetLastError(), "cudaEventCreate"); break; }
@@ -205,7 +238,7 @@ int create_common(sched_ctx** out, int B, int n, const int32_t* s, const int32_t
             e2 = cudaFuncSetAttribute(k3_eval_orders<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn); \
             e3 = cudaFuncSetAttribute(k3_eval_policy<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn); \
             e4 = cudaFuncSetAttribute(k3_base_run<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn)
-            KV_DISPATCH_NIT(h->nit, SETATTR);
+            KV_DISPATCH_SIM(h, SETATTR);
 #undef SETATTR
             if (e1 != cudaSuccess || e2 != cudaSuccess || e3 != cudaSuccess || e4 != cudaSuccess) {
                 rc = kv_cuda_fail(cudaGetLastError(), "cudaFuncSetAttribute(MaxDynamicSharedMemorySize)"); break;
@@ -226,10 +259,10 @@ int ensure_base(sched_ctx* h) {
     const int n = h->n;
     k3_gather_table<<<(n + 255) / 256, 256, 0, h->stream>>>(h->d_tbl_id, h->d_order, n, h->d_tbl_base);
     KV_TRY(check_launch(h));
-#define RUN(N) k3_base_run<N><<<1, 32, (size_t)h->L * sizeof(int), h->stream>>>(                    \
+#define RUN(N) k3_base_run<N><<<1, 32, (size_t)h->L * sizeof(int), h->stream>>>(                   \
         h->d_tbl_base, n, h->L, (int)h->M, h->snap_stride, h->d_snap_ring, h->d_snap_hdr,            \
         h->d_base_starts, h->d_base_tel, h->d_status)
-    KV_DISPATCH_NIT(h->nit, RUN);
+    KV_DISPATCH_SIM(h, RUN);
 #undef RUN
     KV_TRY(check_launch(h));
     h->base_ready = true;
@@ -237,7 +270,8 @@ int ensure_base(sched_ctx* h) {
 }
 
 int k3_grid(const sched_ctx* h, i64 count) {
-    i64 ctas = (count + K3_WARPS - 1) / K3_WARPS;
+    const int w = k3_warps(h);
+    i64 ctas = (count + w - 1) / w;
     if (ctas > h->sm_count) ctas = h->sm_count;
     if (ctas < 1) ctas = 1;
     return (int)ctas;
@@ -261,8 +295,8 @@ int launch_moves(sched_ctx* h, int mode, const i64* codes, i64 first, u64 seed, 
     p.counter = h->d_counter; p.status = h->d_status;
     KV_CUDA(cudaMemsetAsync(h->d_counter, 0, sizeof(unsigned), h->stream));
     KV_CUDA(cudaEventRecord(h->ev_k3_begin, h->stream));
-#define RUN(N) k3_eval_moves<N><<<k3_grid(h, count), K3_THREADS, smem, h->stream>>>(p)
-    KV_DISPATCH_NIT(h->nit, RUN);
+#define RUN(N) k3_eval_moves<N><<<k3_grid(h, count), k3_warps(h) * 32, smem, h->stream>>>(p)
+    KV_DISPATCH_SIM(h, RUN);
 #undef RUN
     KV_TRY(check_launch(h));
     KV_CUDA(cudaEventRecord(h->ev_k3_end, h->stream));
@@ -360,14 +394,15 @@ int sched_eval_batch_dev(sched_handle h, int kind, int64_t count, const void* ca
     if (count >= (1ll << 31)) return SCHED_E_UNSUPPORTED;
     const int n = h->n;
     if (kind == SCHED_CAND_POLICY) {
-        const size_t smem = (size_t)(n + 1) * 16 + (size_t)n * 8 + (size_t)n * 16 + (size_t)(n + 2) * 4 + (size_t)h->L * 4;
+        const size_t smem = (size_t)(n + 1) * 16 + (size_t)n * 8 + (size_t)n * 16 + (size_t)(n + 2) * 4 +
+                            (h->nreg > 0 ? 0 : (size_t)h->L * 4);
         if (smem > (size_t)h->smem_optin - 2048) return SCHED_E_UNSUPPORTED;
         const i64 ctas = (i64)h->B * count;
         if (ctas >= (1ll << 31)) return SCHED_E_UNSUPPORTED;
 #define RUN(N) k3_eval_policy<N><<<(unsigned)ctas, 32, smem, h->stream>>>(h->d_s, h->d_o, n, h->L, (int)h->M, \
                                                                   (const int*)candidates, (int)count,        \
                                                                   (i64*)tel_out, starts_out, h->d_status)
-        KV_DISPATCH_NIT(h->nit, RUN);
+        KV_DISPATCH_SIM(h, RUN);
 #undef RUN
         KV_TRY(check_launch(h));
         h->evaluations += ctas;
@@ -391,8 +426,8 @@ int sched_eval_batch_dev(sched_handle h, int kind, int64_t count, const void* ca
         p.counter = h->d_counter; p.status = h->d_status;
         KV_CUDA(cudaMemsetAsync(h->d_counter, 0, sizeof(unsigned), h->stream));
         KV_CUDA(cudaEventRecord(h->ev_k3_begin, h->stream));
-#define RUN(N) k3_eval_orders<N><<<k3_grid(h, count), K3_THREADS, smem, h->stream>>>(p)
-        KV_DISPATCH_NIT(h->nit, RUN);
+#define RUN(N) k3_eval_orders<N><<<k3_grid(h, count), k3_warps(h) * 32, smem, h->stream>>>(p)
+        KV_DISPATCH_SIM(h, RUN);
 #undef RUN
         KV_TRY(check_launch(h));
         KV_CUDA(cudaEventRecord(h->ev_k3_end, h->stream));
@@ -421,11 +456,16 @@ int sched_eval_batch_dev(sched_handle h, int kind, int64_t count, const void* ca
         KV_TRY(check_launch(h));
         StartsEvalParams p;
         memset(&p, 0, sizeof(p));
-        p.n = n; p.L = h->L; p.M = (int)h->M; p.tbl_id = h->d_tbl_id;
+        p.n = n; p.L = (h->omax + 8 + 31) & ~31; p.M = (int)h->M; p.tbl_id = h->d_tbl_id;
         p.starts = (const int*)candidates; p.sorted_ids = va; p.count = count;
         p.tel_out = (i64*)tel_out; p.feasible_out = feasible_out; p.counter = h->d_counter;
         KV_CUDA(cudaMemsetAsync(h->d_counter, 0, sizeof(unsigned), h->stream));
-        k3_check_starts<<<k3_grid(h, count), K3_THREADS, (size_t)K3_WARPS * h->L * sizeof(int), h->stream>>>(p);
+        int sw = (int)(((size_t)h->smem_optin - 2048) / ((size_t)p.L * sizeof(int)));
+        if (sw > K3S_WARPS) sw = K3S_WARPS;
+        if (sw < 1) return SCHED_E_UNSUPPORTED;
+        const i64 sctas = (count + sw - 1) / sw;
+        k3_check_starts<<<(unsigned)(sctas < h->sm_count ? sctas : h->sm_count), sw * 32,
+                          (size_t)sw * p.L * sizeof(int), h->stream>>>(p);
         KV_TRY(check_launch(h));
         h->evaluations += count;
         return SCHED_OK;

@@ -19,9 +19,9 @@
 #include "common.cuh"
 #include "k2_fmetric.cuh"
 #include "sim.cuh"
+#include "sim_reg.cuh"
 
-#define K3_WARPS 16
-#define K3_THREADS (K3_WARPS * 32)
+#define K3S_WARPS 16                       // warps per CTA of the start-time checker
 
 // ------------------------------------------------------------------------------------------------
 // Bulk copy global -> shared with a bounded wait.  bytes is a multiple of 16, both addresses are
@@ -92,18 +92,18 @@ __global__ void k3_iota(int* a, int n) {
 
 // ------------------------------------------------------------------------------------------------
 // Base run: positions 0 .. n-1 of the base order; snapshot idx holds the state in front of
-// position idx * stride.  One warp.  Dynamic shared memory: L ints.
+// position idx * stride.  One warp.  Dynamic shared memory: L ints (shared-memory simulator only).
 // ------------------------------------------------------------------------------------------------
-template <int NIT>
+template <class SIM>
 __global__ void __launch_bounds__(32)
 k3_base_run(const int2* __restrict__ tbl_base, int n, int L, int M, int stride,
             int* __restrict__ snap_ring, SnapHeader* __restrict__ snap_hdr,
             int* __restrict__ base_starts_pos, i64* __restrict__ base_tel, int* status) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    int* ring = (int*)smem_raw;
     const int lane = threadIdx.x;
-    SimState st;
-    sim_reset(ring, L, st, lane);
+    SIM sim;
+    sim.attach((int*)smem_raw, L);
+    sim.reset(lane);
     for (int q0 = 0; q0 < n; q0 += 32) {
         const int qq = q0 + lane;
         int2 so = qq < n ? tbl_base[qq] : make_int2(1, 1);
@@ -112,19 +112,14 @@ k3_base_run(const int2* __restrict__ tbl_base, int n, int L, int M, int stride,
             const int q = q0 + k;
             if (q % stride == 0) {
                 const int idx = q / stride;
-                for (int r = lane; r < L; r += 32) snap_ring[(size_t)idx * L + r] = ring[r];
-                if (lane == 0) {
-                    SnapHeader h; h.t = st.t; h.hz = st.hz;
-                    h.tel_lo = (int)(st.tel & 0xffffffffll); h.tel_hi = (int)(st.tel >> 32);
-                    snap_hdr[idx] = h;
-                }
+                sim.store(snap_ring + (size_t)idx * L, snap_hdr + idx, lane);
             }
             const int s = __shfl_sync(KV_FULL, so.x, k), o = __shfl_sync(KV_FULL, so.y, k);
-            const int p = sim_admit<NIT>(ring, L, M, st, s, o, lane, status);
+            const int p = sim.admit(s, o, M, lane, status);
             if (lane == 0) base_starts_pos[q] = p;
         }
     }
-    if (lane == 0) *base_tel = st.tel;
+    if (lane == 0) *base_tel = sim.total();
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -151,8 +146,8 @@ struct MoveEvalParams {
     int* status;
 };
 
-template <int NIT>
-__global__ void __launch_bounds__(K3_THREADS, 1)
+template <class SIM>
+__global__ void __launch_bounds__(SIM::kWarps * 32, 1)
 k3_eval_moves(const MoveEvalParams p) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     __shared__ u64 mbar;
@@ -165,8 +160,9 @@ k3_eval_moves(const MoveEvalParams p) {
         tbl = (const int2*)smem_raw;
         ring_off = (p.table_bytes + 127) & ~(size_t)127;
     }
-    int* ring = (int*)(smem_raw + ring_off) + (size_t)warp * p.L;
     const int n = p.n, L = p.L, M = p.M;
+    SIM sim;
+    sim.attach((int*)(smem_raw + ring_off) + (size_t)warp * L, L);
 
     for (;;) {
         unsigned c32 = 0;
@@ -181,13 +177,7 @@ k3_eval_moves(const MoveEvalParams p) {
         const int idx = first_pos / p.stride;
         const int q_start = idx * p.stride;
         // restore the base run's state in front of q_start
-        const int* src = p.snap_ring + (size_t)idx * L;
-        for (int r = lane; r < L; r += 32) ring[r] = src[r];
-        const SnapHeader h = p.snap_hdr[idx];
-        SimState st;
-        st.t = h.t; st.hz = h.hz; st.tr = h.t % L;
-        st.tel = ((i64)h.tel_hi << 32) | (i64)(unsigned)h.tel_lo;
-        __syncwarp();
+        sim.load(p.snap_ring + (size_t)idx * L, p.snap_hdr[idx], lane);
         int* starts = p.starts_out ? p.starts_out + (size_t)c * n : nullptr;
         if (starts)
             for (int q = lane; q < q_start; q += 32) starts[p.base_order[q]] = p.base_starts_pos[q];
@@ -203,11 +193,11 @@ k3_eval_moves(const MoveEvalParams p) {
             const int cnt = min(32, n - q0);
             for (int k = 0; k < cnt; ++k) {
                 const int s = __shfl_sync(KV_FULL, so.x, k), o = __shfl_sync(KV_FULL, so.y, k);
-                const int pstart = sim_admit<NIT>(ring, L, M, st, s, o, lane, p.status);
+                const int pstart = sim.admit(s, o, M, lane, p.status);
                 if (starts && lane == k) starts[id] = pstart;
             }
         }
-        if (lane == 0) p.tel_out[c] = st.tel;
+        if (lane == 0) p.tel_out[c] = sim.total();
     }
 }
 
@@ -227,8 +217,8 @@ struct OrderEvalParams {
     int* status;
 };
 
-template <int NIT>
-__global__ void __launch_bounds__(K3_THREADS, 1)
+template <class SIM>
+__global__ void __launch_bounds__(SIM::kWarps * 32, 1)
 k3_eval_orders(const OrderEvalParams p) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     __shared__ u64 mbar;
@@ -241,8 +231,9 @@ k3_eval_orders(const OrderEvalParams p) {
         tbl = (const int2*)smem_raw;
         ring_off = (p.table_bytes + 127) & ~(size_t)127;
     }
-    int* ring = (int*)(smem_raw + ring_off) + (size_t)warp * p.L;
     const int n = p.n, L = p.L, M = p.M;
+    SIM sim;
+    sim.attach((int*)(smem_raw + ring_off) + (size_t)warp * L, L);
     for (;;) {
         unsigned c32 = 0;
         if (lane == 0) c32 = atomicAdd(p.counter, 1u);
@@ -250,8 +241,7 @@ k3_eval_orders(const OrderEvalParams p) {
         if (c >= p.count) break;
         const int* ord = p.orders + (size_t)c * n;
         int* starts = p.starts_out ? p.starts_out + (size_t)c * n : nullptr;
-        SimState st;
-        sim_reset(ring, L, st, lane);
+        sim.reset(lane);
         for (int q0 = 0; q0 < n; q0 += 32) {
             const int qq = q0 + lane;
             int2 so = make_int2(1, 1);
@@ -260,18 +250,18 @@ k3_eval_orders(const OrderEvalParams p) {
             const int cnt = min(32, n - q0);
             for (int k = 0; k < cnt; ++k) {
                 const int s = __shfl_sync(KV_FULL, so.x, k), o = __shfl_sync(KV_FULL, so.y, k);
-                const int pstart = sim_admit<NIT>(ring, L, M, st, s, o, lane, p.status);
+                const int pstart = sim.admit(s, o, M, lane, p.status);
                 if (starts && lane == k) starts[id] = pstart;
             }
         }
-        if (lane == 0) p.tel_out[c] = st.tel;
+        if (lane == 0) p.tel_out[c] = sim.total();
     }
 }
 
 // ------------------------------------------------------------------------------------------------
 // Policy sweep: grid = B * P single-warp CTAs; CTA (b, k) evaluates instance b under policies[k].
-// Dynamic shared memory: int ring[L]; i64 P[n+1], O[n+1]; u64 key[n]; int s[n], o[n], ord[n], tmp[n],
-// boff[n+2].
+// Dynamic shared memory: int ring[L] (shared-memory simulator only; L = 0 otherwise); i64 P[n+1],
+// O[n+1]; u64 key[n]; int s[n], o[n], ord[n], tmp[n], boff[n+2].
 // ------------------------------------------------------------------------------------------------
 __device__ __forceinline__ void k3_rank_sort(const u64* key, const int* ids_in, int* ids_out, int lo, int hi, int lane) {
     // ids_out[lo + rank] = ids_in[e]; rank by (key, position) -- keys carry their own tie-breakers
@@ -287,7 +277,7 @@ __device__ __forceinline__ void k3_rank_sort(const u64* key, const int* ids_in, 
     __syncwarp();
 }
 
-template <int NIT>
+template <class SIM>
 __global__ void __launch_bounds__(32)
 k3_eval_policy(const int* __restrict__ s_all, const int* __restrict__ o_all, int n, int L, int M,
                const int* __restrict__ policies, int num_policies,
@@ -297,7 +287,7 @@ k3_eval_policy(const int* __restrict__ s_all, const int* __restrict__ o_all, int
     const int b = blockIdx.x / num_policies, kpol = blockIdx.x % num_policies;
     const int policy = policies[kpol];
     int* ring = (int*)smem_raw;                       // first: 16-byte aligned for the vector loads
-    i64* P = (i64*)(ring + L);                        // L is a multiple of 4
+    i64* P = (i64*)(ring + (SIM::kUsesSmem ? L : 0)); // L is a multiple of 4
     i64* O = P + (n + 1);
     u64* key = (u64*)(O + (n + 1));
     int* s = (int*)(key + n);
@@ -341,15 +331,16 @@ k3_eval_policy(const int* __restrict__ s_all, const int* __restrict__ o_all, int
             for (int bi = 0; bi < nb; ++bi) k3_rank_sort(key, tmp, ord, boff[bi], boff[bi + 1], lane);
         }
     }
-    SimState st;
-    sim_reset(ring, L, st, lane);
+    SIM sim;
+    sim.attach(ring, L);
+    sim.reset(lane);
     int* starts = starts_out ? starts_out + ((size_t)b * num_policies + kpol) * n : nullptr;
     for (int q = 0; q < n; ++q) {
         const int id = ord[q];
-        const int pstart = sim_admit<NIT>(ring, L, M, st, s[id], o[id], lane, status);
+        const int pstart = sim.admit(s[id], o[id], M, lane, status);
         if (starts && lane == 0) starts[id] = pstart;
     }
-    if (lane == 0) tel_out[(size_t)b * num_policies + kpol] = st.tel;
+    if (lane == 0) tel_out[(size_t)b * num_policies + kpol] = sim.total();
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -369,7 +360,7 @@ struct StartsEvalParams {
     unsigned int* counter;
 };
 
-__global__ void __launch_bounds__(K3_THREADS, 1)
+__global__ void __launch_bounds__(K3S_WARPS * 32, 1)
 k3_check_starts(const StartsEvalParams p) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;

@@ -26,9 +26,10 @@
 // stay fine when p grows, so only the cells that enter the window on the right are looked at again.
 //
 // Two code shapes with identical results:
-//   sim_admit<NIT>, NIT >= 1: the window (<= 128*NIT + 3 cells) is loaded once with 16-byte shared
-//     loads into registers, checked, and written back -- one read and one write per cell;
-//   sim_admit<0>: any window length, cells are re-read by the write pass.
+//   cached (NIT >= 1, windows of at most 32*NIT full 16-byte groups): the window is loaded once
+//     with 16-byte shared loads into registers, checked, and written back -- one read and one
+//     write per cell;
+//   streamed (longer windows, or NIT = 0): any window length, cells are re-read by the write pass.
 #pragma once
 
 #include "common.cuh"
@@ -104,10 +105,10 @@ __device__ __forceinline__ int sim_admit(int* __restrict__ ring, int L, int M, S
     const int kw = s + 1;                            // ramp value at the window start
     int delta = 0;
 
-    if (NIT > 0) {
-        const int h = (4 - (tr & 3)) & 3;            // L is a multiple of 4: t and tr agree mod 4
-        const int hc = o < h ? o : h;                // head cells
-        const int nbody = (o - hc) >> 2;             // full groups
+    const int h = (4 - (tr & 3)) & 3;                // L is a multiple of 4: t and tr agree mod 4
+    const int hc = o < h ? o : h;                    // head cells
+    const int nbody = (o - hc) >> 2;                 // full groups
+    if (NIT > 0 && nbody <= 32 * NIT) {
         const int tc = (o - hc) & 3;                 // tail cells
         const int nit = (nbody + 31) >> 5;
         const int ab = kv_wrap1(tr + hc, L);         // ring index of the first body cell (16-byte aligned)
@@ -213,10 +214,41 @@ __device__ __forceinline__ int sim_admit(int* __restrict__ ring, int L, int M, S
     return p;
 }
 
+// The shared-memory simulator behind the interface the kernels use (see RegSim for the other one).
+template <int NIT>
+struct SmemSim {
+    static constexpr bool kUsesSmem = true;
+    static constexpr int kWarps = 24;                 // warps per CTA of the persistent kernels
+    int* ring;
+    int L;
+    SimState st;
+
+    __device__ __forceinline__ void attach(int* ring_, int L_) { ring = ring_; L = L_; }
+    __device__ __forceinline__ void reset(int lane) { sim_reset(ring, L, st, lane); }
+    __device__ __forceinline__ void load(const int* __restrict__ snap, const SnapHeader& h, int lane) {
+        for (int r = lane; r < L; r += 32) ring[r] = snap[r];
+        st.t = h.t; st.hz = h.hz; st.tr = h.t % L;
+        st.tel = ((i64)h.tel_hi << 32) | (i64)(unsigned)h.tel_lo;
+        __syncwarp();
+    }
+    __device__ __forceinline__ void store(int* __restrict__ snap, SnapHeader* hdr, int lane) const {
+        for (int r = lane; r < L; r += 32) snap[r] = ring[r];
+        if (lane == 0) {
+            SnapHeader h; h.t = st.t; h.hz = st.hz;
+            h.tel_lo = (int)(st.tel & 0xffffffffll); h.tel_hi = (int)(st.tel >> 32);
+            *hdr = h;
+        }
+    }
+    __device__ __forceinline__ int admit(int s, int o, int M, int lane, int* status) {
+        return sim_admit<NIT>(ring, L, M, st, s, o, lane, status);
+    }
+    __device__ __forceinline__ i64 total() const { return st.tel; }
+};
+
 // Number of 128-cell rounds a handle's longest window needs (0: use the streamed form).
 static inline int sim_pick_nit(int omax) {
     const int need = (omax / 4 + 31) / 32;            // full 4-cell groups of the longest window
     const int sizes[] = {1, 2, 4, 8};
     for (int k = 0; k < 4; ++k) if (need <= sizes[k]) return sizes[k];
-    return 0;
+    return 8;                                         // longer windows take the streamed form
 }
