@@ -17,39 +17,33 @@
 //      t moves, and step 1 is repeated at the new start (it also covers the cells that entered the
 //      window on the right);
 //   3. the ramp s+1+r is added to the window.
-// No shared memory, no address arithmetic, no loads or stores: two integer instructions per cell
-// chunk and admission in the common case.
+// No shared memory, no address arithmetic, no loads or stores: two integer instructions per
+// 32-cell chunk and admission in the common case.
 #pragma once
 
 #include "common.cuh"
 
-// Runs BODY(c) for c = nch-1 down to 1 through a jump table (a switch that falls through), so that
-// only the registers of the window are touched: the cases are entry points into straight-line
-// code, which keeps the compiler from predicating all NREG bodies.
-#define KV_RS_CASE(c, BODY) case (c) + 1: if constexpr ((c) < NREG) { BODY(c) } [[fallthrough]];
-#define KV_RS_CHUNKS(nch, BODY)                                                                       \
-    switch (nch) {                                                                                    \
-        KV_RS_CASE(32, BODY) KV_RS_CASE(31, BODY) KV_RS_CASE(30, BODY) KV_RS_CASE(29, BODY)           \
-        KV_RS_CASE(28, BODY) KV_RS_CASE(27, BODY) KV_RS_CASE(26, BODY) KV_RS_CASE(25, BODY)           \
-        KV_RS_CASE(24, BODY) KV_RS_CASE(23, BODY) KV_RS_CASE(22, BODY) KV_RS_CASE(21, BODY)           \
-        KV_RS_CASE(20, BODY) KV_RS_CASE(19, BODY) KV_RS_CASE(18, BODY) KV_RS_CASE(17, BODY)           \
-        KV_RS_CASE(16, BODY) KV_RS_CASE(15, BODY) KV_RS_CASE(14, BODY) KV_RS_CASE(13, BODY)           \
-        KV_RS_CASE(12, BODY) KV_RS_CASE(11, BODY) KV_RS_CASE(10, BODY) KV_RS_CASE(9, BODY)            \
-        KV_RS_CASE(8, BODY) KV_RS_CASE(7, BODY) KV_RS_CASE(6, BODY) KV_RS_CASE(5, BODY)               \
-        KV_RS_CASE(4, BODY) KV_RS_CASE(3, BODY) KV_RS_CASE(2, BODY) KV_RS_CASE(1, BODY)               \
-        default: break;                                                                               \
+// The passes over the window are specialised on a bucket (KLO, KHI] of the chunk count nch, chosen
+// by a short tree of warp-uniform branches: chunks 1 .. KLO-1 are certainly inside the window (one
+// instruction each), chunks KLO .. KHI-1 are masked by lane, and no other register is touched.
+// STMT(KLO, KHI) is expanded once per bucket.
+#define KV_RS_BUCKETS(nch, STMT)                                                                        \
+    if (nch <= 8) {                                                                                     \
+        if (nch <= 4) { if (nch <= 2) { STMT(0, 2) } else { STMT(2, 4) } }                              \
+        else { if (nch <= 6) { STMT(4, 6) } else { STMT(6, 8) } }                                       \
+    } else if (nch <= 16) {                                                                             \
+        if (nch <= 12) { if (nch <= 10) { STMT(8, 10) } else { STMT(10, 12) } } else { STMT(12, 16) }   \
+    } else {                                                                                            \
+        if (nch <= 24) { STMT(16, 24) } else { STMT(24, 33) }                                           \
     }
 
 template <int NREG>
 struct RegSim {
-    static_assert(NREG >= 2 && NREG <= 33, "the chunk switch covers up to 33 registers");
+    static_assert(NREG >= 2 && NREG <= 33, "the bucket tree covers up to 33 registers");
     static constexpr int kCells = 32 * NREG;
     static constexpr bool kUsesSmem = false;
-#ifndef KV_REG33_WARPS
-#define KV_REG33_WARPS 16
-#endif
     // warps per CTA of the persistent kernels, limited by the register file (64K / threads)
-    static constexpr int kWarps = NREG > 17 ? KV_REG33_WARPS : (NREG > 9 ? 24 : 32);
+    static constexpr int kWarps = NREG > 17 ? 28 : 32;
     int R[NREG];
     int t;
     i64 tel;
@@ -88,24 +82,48 @@ struct RegSim {
         R[NREG - 1] = first;
     }
 
+    // rl = window offset of this lane's cell of R[0]; the cell of R[c] is inside the window iff
+    // 32 c < ol (and rl >= 0 for c = 0), with ol = o - rl.
+    template <int KLO, int KHI>
+    __device__ __forceinline__ int pass_max(int rl, int ol) const {
+        int v = (rl >= 0 && ol > 0) ? R[0] : -1;
+#pragma unroll
+        for (int c = 1; c < KHI; ++c) v = max(v, (c < KLO || 32 * c < ol) ? R[c] : -1);
+        return v;
+    }
+    template <int KLO, int KHI>
+    __device__ __forceinline__ void pass_add(int rl, int ol, int k0) {
+        if (rl >= 0 && ol > 0) R[0] += k0;
+#pragma unroll
+        for (int c = 1; c < KHI; ++c)
+            if (c < KLO || 32 * c < ol) R[c] += k0 + 32 * c;
+    }
+    template <int KLO, int KHI>
+    __device__ __forceinline__ int pass_need(int rl, int ol, int kadm) const {
+        int need = (rl >= 0 && ol > 0) ? min(R[0] + kadm, rl + 1) : 0;
+#pragma unroll
+        for (int c = 1; c < KHI; ++c)
+            if (c < KLO || 32 * c < ol) need = max(need, min(R[c] + kadm, rl + 1 + 32 * c));
+        return need;
+    }
+
     // Admit one request; returns its start.  All 32 lanes call this with identical (s, o).
     __device__ __forceinline__ int admit(int s, int o, int M, int lane, int* status) {
         int kadm = s + 1 - M - t;                      // V + kadm > 0  <=>  the cell is over budget
         for (int guard = 0;; ++guard) {
             const int tm = t & 31;
-            const int rl = lane - tm;                  // window offset of this lane's cell of R[0]
-            const int ol = o - rl;                     // cell of R[c] is inside the window iff 32 c < ol
+            const int rl = lane - tm;
+            const int ol = o - rl;
             const int nch = (tm + o + 31) >> 5;
-            const bool in0 = rl >= 0 && ol > 0;
-            int vmax = in0 ? R[0] : -1;
-#define KV_RS_MAX(c) vmax = max(vmax, 32 * (c) < ol ? R[c] : -1);
-            KV_RS_CHUNKS(nch, KV_RS_MAX)
+            int vmax = -1;
+#define KV_RS_MAX(A, B) vmax = pass_max<A, (B < NREG ? B : NREG)>(rl, ol);
+            KV_RS_BUCKETS(nch, KV_RS_MAX)
 #undef KV_RS_MAX
             vmax = kv_warp_max(vmax);
             if (vmax + kadm <= 0) break;
-            int need = in0 ? min(R[0] + kadm, rl + 1) : 0;
-#define KV_RS_NEED(c) if (32 * (c) < ol) need = max(need, min(R[c] + kadm, rl + 1 + 32 * (c)));
-            KV_RS_CHUNKS(nch, KV_RS_NEED)
+            int need = 0;
+#define KV_RS_NEED(A, B) need = pass_need<A, (B < NREG ? B : NREG)>(rl, ol, kadm);
+            KV_RS_BUCKETS(nch, KV_RS_NEED)
 #undef KV_RS_NEED
             int delta = kv_warp_max(need);             // >= 1: the worst cell alone asks for it
             kadm -= delta;
@@ -125,9 +143,8 @@ struct RegSim {
         const int ol = o - rl;
         const int nch = (tm + o + 31) >> 5;
         const int k0 = s + 1 + rl;                     // ramp value of this lane's cell of R[0]
-        if (rl >= 0 && ol > 0) R[0] += k0;
-#define KV_RS_ADD(c) if (32 * (c) < ol) R[c] += k0 + 32 * (c);
-        KV_RS_CHUNKS(nch, KV_RS_ADD)
+#define KV_RS_ADD(A, B) pass_add<A, (B < NREG ? B : NREG)>(rl, ol, k0);
+        KV_RS_BUCKETS(nch, KV_RS_ADD)
 #undef KV_RS_ADD
         tel += t + o;
         return t;
