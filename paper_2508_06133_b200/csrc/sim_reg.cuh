@@ -87,8 +87,12 @@ struct RegSim {
     template <int KLO, int KHI>
     __device__ __forceinline__ int pass_max(int rl, int ol) const {
         int v = (rl >= 0 && ol > 0) ? R[0] : -1;
+        constexpr int KI = KLO < KHI ? KLO : KHI;      // chunks 1 .. KI-1 need no mask
 #pragma unroll
-        for (int c = 1; c < KHI; ++c) v = max(v, (c < KLO || 32 * c < ol) ? R[c] : -1);
+        for (int c = 1; c + 1 < KI; c += 2) v = __vimax3_s32(v, R[c], R[c + 1]);
+        if constexpr (KI >= 2 && ((KI - 1) & 1)) v = max(v, R[KI - 1]);
+#pragma unroll
+        for (int c = (KI > 1 ? KI : 1); c < KHI; ++c) v = max(v, (32 * c < ol) ? R[c] : -1);
         return v;
     }
     template <int KLO, int KHI>
@@ -103,45 +107,68 @@ struct RegSim {
         int need = (rl >= 0 && ol > 0) ? min(R[0] + kadm, rl + 1) : 0;
 #pragma unroll
         for (int c = 1; c < KHI; ++c)
-            if (c < KLO || 32 * c < ol) need = max(need, min(R[c] + kadm, rl + 1 + 32 * c));
+            if (c < KLO || 32 * c < ol) need = max(need, __viaddmin_s32(R[c], kadm, rl + 1 + 32 * c));
         return need;
+    }
+
+    // Rounds t .. t+delta-1 are over: their cells are re-labelled for the rounds L later and the
+    // registers rotate once per 32-round boundary crossed.  The rotation sits behind a real branch
+    // (it is rare; as predicated moves it would cost NREG instructions on every call).
+    __device__ __forceinline__ void advance(int delta, int lane) {
+        const int tm = t & 31, rl = lane - tm;
+        const int step = min(delta, 32 - tm);
+        if (rl >= 0 && rl < step) R[0] = t + rl + kCells;
+        t += step;
+        delta -= step;
+        if (tm + step == 32) {
+            asm volatile("" ::: "memory");
+            rotate();
+            while (delta >= 32) { R[0] = t + lane + kCells; t += 32; delta -= 32; rotate(); }
+            if (lane < delta) R[0] = t + lane + kCells;
+            t += delta;
+        }
     }
 
     // Admit one request; returns its start.  All 32 lanes call this with identical (s, o).
     __device__ __forceinline__ int admit(int s, int o, int M, int lane, int* status) {
         int kadm = s + 1 - M - t;                      // V + kadm > 0  <=>  the cell is over budget
+        {   // common case: the request fits at t -- test and ramp add inside one bucket dispatch
+            const int tm = t & 31, rl = lane - tm, ol = o - rl, nch = (tm + o + 31) >> 5;
+#define KV_RS_FAST(A, B)                                                           \
+            {                                                                      \
+                int vmax = pass_max<A, (B < NREG ? B : NREG)>(rl, ol);             \
+                vmax = kv_warp_max(vmax);                                          \
+                if (vmax + kadm <= 0) {                                            \
+                    pass_add<A, (B < NREG ? B : NREG)>(rl, ol, s + 1 + rl);        \
+                    tel += t + o;                                                  \
+                    return t;                                                      \
+                }                                                                  \
+            }
+            KV_RS_BUCKETS(nch, KV_RS_FAST)
+#undef KV_RS_FAST
+        }
+        // blocked at t: skip ahead, re-test at the new start (this also covers the cells that
+        // entered the window on the right), repeat until the request fits
         for (int guard = 0;; ++guard) {
-            const int tm = t & 31;
-            const int rl = lane - tm;
-            const int ol = o - rl;
-            const int nch = (tm + o + 31) >> 5;
-            int vmax = -1;
+            const int tm = t & 31, rl = lane - tm, ol = o - rl, nch = (tm + o + 31) >> 5;
+            if (guard > 0) {
+                int vmax = -1;
 #define KV_RS_MAX(A, B) vmax = pass_max<A, (B < NREG ? B : NREG)>(rl, ol);
-            KV_RS_BUCKETS(nch, KV_RS_MAX)
+                KV_RS_BUCKETS(nch, KV_RS_MAX)
 #undef KV_RS_MAX
-            vmax = kv_warp_max(vmax);
-            if (vmax + kadm <= 0) break;
+                vmax = kv_warp_max(vmax);
+                if (vmax + kadm <= 0) break;
+            }
             int need = 0;
 #define KV_RS_NEED(A, B) need = pass_need<A, (B < NREG ? B : NREG)>(rl, ol, kadm);
             KV_RS_BUCKETS(nch, KV_RS_NEED)
 #undef KV_RS_NEED
-            int delta = kv_warp_max(need);             // >= 1: the worst cell alone asks for it
+            const int delta = kv_warp_max(need);       // >= 1: the worst cell alone asks for it
             kadm -= delta;
-            // rounds t .. t+delta-1 are over: re-label their cells for the rounds L later
-            while (delta > 0) {
-                const int tm2 = t & 31;
-                const int step = min(delta, 32 - tm2);
-                if (lane >= tm2 && lane < tm2 + step) R[0] = t - tm2 + lane + kCells;
-                t += step;
-                delta -= step;
-                if (tm2 + step == 32) rotate();
-            }
+            advance(delta, lane);
             if (guard > kCells) { if (lane == 0) atomicExch(status, KV_DEV_LOOP_CAP); break; }
         }
-        const int tm = t & 31;
-        const int rl = lane - tm;
-        const int ol = o - rl;
-        const int nch = (tm + o + 31) >> 5;
+        const int tm = t & 31, rl = lane - tm, ol = o - rl, nch = (tm + o + 31) >> 5;
         const int k0 = s + 1 + rl;                     // ramp value of this lane's cell of R[0]
 #define KV_RS_ADD(A, B) pass_add<A, (B < NREG ? B : NREG)>(rl, ol, k0);
         KV_RS_BUCKETS(nch, KV_RS_ADD)
