@@ -43,7 +43,10 @@ struct RegSim {
     static constexpr int kCells = 32 * NREG;
     static constexpr bool kUsesSmem = false;
     // warps per CTA of the persistent kernels, limited by the register file (64K / threads)
-    static constexpr int kWarps = NREG > 17 ? 28 : 32;
+#ifndef KV_REG33_WARPS
+#define KV_REG33_WARPS 32
+#endif
+    static constexpr int kWarps = NREG > 17 ? KV_REG33_WARPS : 32;
     int R[NREG];
     int t;
     i64 tel;
@@ -130,51 +133,36 @@ struct RegSim {
     }
 
     // Admit one request; returns its start.  All 32 lanes call this with identical (s, o).
+    // Each turn of the loop is one bucket dispatch at the current t: test; if the request fits, add
+    // its ramp and return; otherwise compute the advance the window asks for, move t, and try again
+    // (the next test also covers the cells that entered the window on the right).
     __device__ __forceinline__ int admit(int s, int o, int M, int lane, int* status) {
         int kadm = s + 1 - M - t;                      // V + kadm > 0  <=>  the cell is over budget
-        {   // common case: the request fits at t -- test and ramp add inside one bucket dispatch
-            const int tm = t & 31, rl = lane - tm, ol = o - rl, nch = (tm + o + 31) >> 5;
-#define KV_RS_FAST(A, B)                                                           \
-            {                                                                      \
-                int vmax = pass_max<A, (B < NREG ? B : NREG)>(rl, ol);             \
-                vmax = kv_warp_max(vmax);                                          \
-                if (vmax + kadm <= 0) {                                            \
-                    pass_add<A, (B < NREG ? B : NREG)>(rl, ol, s + 1 + rl);        \
-                    tel += t + o;                                                  \
-                    return t;                                                      \
-                }                                                                  \
-            }
-            KV_RS_BUCKETS(nch, KV_RS_FAST)
-#undef KV_RS_FAST
+        int delta = 0;
+#define KV_RS_TRY(A, B)                                                            \
+        {                                                                          \
+            int vmax = pass_max<A, (B < NREG ? B : NREG)>(rl, ol);                 \
+            vmax = kv_warp_max(vmax);                                              \
+            if (vmax + kadm <= 0) {                                                \
+                pass_add<A, (B < NREG ? B : NREG)>(rl, ol, s + 1 + rl);            \
+                tel += t + o;                                                      \
+                return t;                                                          \
+            }                                                                      \
+            delta = pass_need<A, (B < NREG ? B : NREG)>(rl, ol, kadm);             \
         }
-        // blocked at t: skip ahead, re-test at the new start (this also covers the cells that
-        // entered the window on the right), repeat until the request fits
-        for (int guard = 0;; ++guard) {
+        {   // common case: the request fits at t
             const int tm = t & 31, rl = lane - tm, ol = o - rl, nch = (tm + o + 31) >> 5;
-            if (guard > 0) {
-                int vmax = -1;
-#define KV_RS_MAX(A, B) vmax = pass_max<A, (B < NREG ? B : NREG)>(rl, ol);
-                KV_RS_BUCKETS(nch, KV_RS_MAX)
-#undef KV_RS_MAX
-                vmax = kv_warp_max(vmax);
-                if (vmax + kadm <= 0) break;
-            }
-            int need = 0;
-#define KV_RS_NEED(A, B) need = pass_need<A, (B < NREG ? B : NREG)>(rl, ol, kadm);
-            KV_RS_BUCKETS(nch, KV_RS_NEED)
-#undef KV_RS_NEED
-            const int delta = kv_warp_max(need);       // >= 1: the worst cell alone asks for it
+            KV_RS_BUCKETS(nch, KV_RS_TRY)
+        }
+        for (int guard = 0;; ++guard) {
+            delta = kv_warp_max(delta);                // >= 1: the worst cell alone asks for it
             kadm -= delta;
             advance(delta, lane);
-            if (guard > kCells) { if (lane == 0) atomicExch(status, KV_DEV_LOOP_CAP); break; }
+            const int tm = t & 31, rl = lane - tm, ol = o - rl, nch = (tm + o + 31) >> 5;
+            KV_RS_BUCKETS(nch, KV_RS_TRY)
+            if (guard > kCells) { if (lane == 0) atomicExch(status, KV_DEV_LOOP_CAP); return t; }
         }
-        const int tm = t & 31, rl = lane - tm, ol = o - rl, nch = (tm + o + 31) >> 5;
-        const int k0 = s + 1 + rl;                     // ramp value of this lane's cell of R[0]
-#define KV_RS_ADD(A, B) pass_add<A, (B < NREG ? B : NREG)>(rl, ol, k0);
-        KV_RS_BUCKETS(nch, KV_RS_ADD)
-#undef KV_RS_ADD
-        tel += t + o;
-        return t;
+#undef KV_RS_TRY
     }
 };
 
