@@ -234,7 +234,8 @@ int create_common(sched_ctx** out, int B, int n, const int32_t* s, const int32_t
             const int dyn = h->smem_optin - 2048;
             cudaError_t e1 = cudaSuccess, e2 = cudaSuccess, e3 = cudaSuccess, e4 = cudaSuccess;
 #define SETATTR(N)                                                                                         \
-            e1 = cudaFuncSetAttribute(k3_eval_moves<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn);  \
+            e1 = cudaFuncSetAttribute(k3_eval_moves<N, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn);  \
+            if (e1 == cudaSuccess) e1 = cudaFuncSetAttribute(k3_eval_moves<N, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn);  \
             e2 = cudaFuncSetAttribute(k3_eval_orders<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn); \
             e3 = cudaFuncSetAttribute(k3_eval_policy<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn); \
             e4 = cudaFuncSetAttribute(k3_base_run<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn)
@@ -295,7 +296,9 @@ int launch_moves(sched_ctx* h, int mode, const i64* codes, i64 first, u64 seed, 
     p.counter = h->d_counter; p.status = h->d_status;
     KV_CUDA(cudaMemsetAsync(h->d_counter, 0, sizeof(unsigned), h->stream));
     KV_CUDA(cudaEventRecord(h->ev_k3_begin, h->stream));
-#define RUN(N) k3_eval_moves<N><<<k3_grid(h, count), k3_warps(h) * 32, smem, h->stream>>>(p)
+#define RUN(N)                                                                                    \
+    if (starts_out) k3_eval_moves<N, true><<<k3_grid(h, count), k3_warps(h) * 32, smem, h->stream>>>(p);  \
+    else k3_eval_moves<N, false><<<k3_grid(h, count), k3_warps(h) * 32, smem, h->stream>>>(p)
     KV_DISPATCH_SIM(h, RUN);
 #undef RUN
     KV_TRY(check_launch(h));

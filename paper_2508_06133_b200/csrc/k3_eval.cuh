@@ -146,7 +146,7 @@ struct MoveEvalParams {
     int* status;
 };
 
-template <class SIM>
+template <class SIM, bool kStarts>
 __global__ void __launch_bounds__(SIM::kWarps * 32, 1)
 k3_eval_moves(const MoveEvalParams p) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -178,8 +178,8 @@ k3_eval_moves(const MoveEvalParams p) {
         const int q_start = idx * p.stride;
         // restore the base run's state in front of q_start
         sim.load(p.snap_ring + (size_t)idx * L, p.snap_hdr[idx], lane);
-        int* starts = p.starts_out ? p.starts_out + (size_t)c * n : nullptr;
-        if (starts)
+        int* starts = kStarts ? p.starts_out + (size_t)c * n : nullptr;
+        if (kStarts)
             for (int q = lane; q < q_start; q += 32) starts[p.base_order[q]] = p.base_starts_pos[q];
         for (int q0 = q_start; q0 < n; q0 += 32) {
             const int qq = q0 + lane;
@@ -188,13 +188,13 @@ k3_eval_moves(const MoveEvalParams p) {
             if (qq < n) {
                 const int bp = kv_map_pos(mv, qq);
                 so = tbl[bp];
-                if (starts) id = p.base_order[bp];
+                if (kStarts) id = p.base_order[bp];
             }
             const int cnt = min(32, n - q0);
             for (int k = 0; k < cnt; ++k) {
                 const int s = __shfl_sync(KV_FULL, so.x, k), o = __shfl_sync(KV_FULL, so.y, k);
                 const int pstart = sim.admit(s, o, M, lane, p.status);
-                if (starts && lane == k) starts[id] = pstart;
+                if (kStarts && lane == k) starts[id] = pstart;
             }
         }
         if (lane == 0) p.tel_out[c] = sim.total();
