@@ -114,6 +114,20 @@ def sampled_move_positions(n, seed, iteration, first, count):
     return (h1 & np.uint64(1)).astype(np.int64), i, j
 
 
+def rank_first_sample(rank: int, count: int) -> int:
+    """Ranks evaluate disjoint, contiguous slices of one sampled neighbourhood: rank r takes the
+    sample indices [r * count, (r + 1) * count)."""
+    return rank * count
+
+
+def max_over_ranks(value: float, dist, device) -> float:
+    """Slowest rank's figure (the time that counts for a job spread over ranks)."""
+    import torch
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
 def run_reference(args, inst, rank):
     """The CPU oracle as it stands, timed on this machine's host cores on a bounded sample per step."""
     if rank != 0:
@@ -194,7 +208,7 @@ def main():
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
         h.sorted_f_dev()
-        h.sweep_dev(count, best, sampled=True, seed=seed, iteration=k, first_code=rank * count)
+        h.sweep_dev(count, best, sampled=True, seed=seed, iteration=k, first_code=rank_first_sample(rank, count))
         e1.record(stream)
         e1.synchronize()
         return e0.elapsed_time(e1), h.last_eval_kernel_ms()
@@ -221,9 +235,7 @@ def main():
     launches1, _ = h.stats()
     total_ms = float(sum(step_ms))
     if world > 1:
-        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+        total_ms = max_over_ranks(total_ms, dist, dev)
     value = world * count * args.steps / (total_ms * 1e-3)
 
     # ---- algorithmic work of the simulator launches: timeline cells that must be updated, i.e.
@@ -232,7 +244,7 @@ def main():
     suffix_o = np.concatenate([np.cumsum(inst.o[order][::-1].astype(np.int64))[::-1], [0]])
     cells = []
     for k in range(args.steps):
-        _, mi, mj = sampled_move_positions(n, seed, args.warmup + k, rank * count, count)
+        _, mi, mj = sampled_move_positions(n, seed, args.warmup + k, rank_first_sample(rank, count), count)
         cells.append(int(suffix_o[np.minimum(mi, mj)].sum()))
     cells_per_launch = float(np.mean(cells))
     kern_s = float(np.mean(kern_ms)) * 1e-3
@@ -282,9 +294,7 @@ def main():
     torch.cuda.synchronize()
     dt = time.perf_counter() - t0
     if world > 1:
-        t = torch.tensor([dt], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        dt = float(t.item())
+        dt = max_over_ranks(dt, dist, dev)
     e2e = {"value": world * count * e2e_steps / dt, "unit": "evals/s",
            "h2d_bytes_per_step": int(8 * n + 8 * count), "d2h_bytes_per_step": int(8 * count + 4 * n + 8),
            "steps": e2e_steps}

@@ -318,3 +318,51 @@ def test_error_paths_on_a_handle():
         assert tel[0] == orc.list_schedule_alg1(s, o, 20, [2, 1, 0])[1]
         launches, evals = h.stats()
         assert launches > 0 and evals >= 1
+
+
+# ------------------------------------------------------------------------------------ full-size configurations
+def test_policy_sweep_full_size_sampled_instances():
+    """4,096 instances x 4 policies in one launch; a sample of instances is re-evaluated by the oracle."""
+    s, o, M = W.policy_sweep()
+    pols = np.array([kv.POLICY_SORTED_F, kv.POLICY_FCFS, kv.POLICY_SOF, kv.POLICY_TOTAL_SIZE], dtype=np.int32)
+    with kv.Scheduler.batch(s, o, M) as h:
+        tel, _, _ = h.eval_batch(kv.CAND_POLICY, pols)
+    assert tel.shape == (4096, 4)
+    for b in list(range(0, 4096, 97)) + [4095]:
+        refs = [orc.sorted_f_prefix(s[b], o[b], M)[0], orc.policy_order(s[b], o[b], orc.FCFS),
+                orc.policy_order(s[b], o[b], orc.SHORTEST_OUTPUT_FIRST), orc.policy_order(s[b], o[b], orc.TOTAL_SIZE_FIRST)]
+        assert tel[b].tolist() == [orc.list_schedule_rounds(s[b], o[b], M, r)[1] for r in refs]
+    # Sorted-F is not worse than FCFS on the bulk of these mixed backlogs
+    assert (tel[:, 0] <= tel[:, 1]).mean() > 0.9
+
+
+def test_heavy_100k_backlog():
+    """n = 100,000, o up to 4,096 (shared-memory simulator, strided snapshots), int64 TELs."""
+    inst = W.heavy_100k()
+    n = inst.n
+    with kv.Scheduler(inst.s, inst.o, inst.M) as h:
+        order, offs, tel = h.sorted_f()
+        r_order, r_offs = orc.sorted_f_prefix(inst.s, inst.o, inst.M)
+        assert (offs == r_offs).all() and (order == r_order).all()
+        p, r_tel, _ = orc.list_schedule_rounds(inst.s, inst.o, inst.M, r_order)
+        assert tel == r_tel
+        fcfs, _, _ = h.eval_batch(kv.CAND_ORDER, np.arange(n, dtype=np.int32)[None, :])
+        assert fcfs[0] == orc.list_schedule_rounds(inst.s, inst.o, inst.M, np.arange(n))[1]
+        assert fcfs[0] > 2 ** 32                                    # beyond 32 bits: TELs are int64
+        total = n * (n - 1) // 2 + n * (n - 1)
+        codes = (W.u64(41, 0, np.arange(6)) % np.uint64(total)).astype(np.int64)
+        codes[0], codes[1] = n * (n - 1) // 2 - 1, total - 1
+        mtel, _, _ = h.eval_batch(kv.CAND_MOVE, codes)
+        assert (mtel == oracle_moves(inst.s, inst.o, inst.M, r_order, codes)).all()
+        final, ftel, done, trace = h.local_search(kv.NBHD_SAMPLED, 2, seed=17, samples_per_iter=1 << 13)
+    assert done == 2 and ftel <= tel
+    cur, cur_tel = r_order, r_tel
+    for it, (m, best) in enumerate(trace):
+        cand = orc.apply_move(cur, *orc.sample_move(n, 17, it, int(m)))
+        assert orc.list_schedule_rounds(inst.s, inst.o, inst.M, cand)[1] == best
+        for mm in (0, 1, (1 << 13) - 1):                           # no sampled move beats the reported best
+            c2 = orc.apply_move(cur, *orc.sample_move(n, 17, it, mm))
+            assert orc.list_schedule_rounds(inst.s, inst.o, inst.M, c2)[1] >= best
+        if best < cur_tel:
+            cur, cur_tel = cand, best
+    assert (final == cur).all() and ftel == cur_tel
