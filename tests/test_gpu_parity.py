@@ -336,6 +336,35 @@ def test_policy_sweep_full_size_sampled_instances():
     assert (tel[:, 0] <= tel[:, 1]).mean() > 0.9
 
 
+def test_mixed_1k_swap_search_to_local_optimum():
+    """Sorted-F then 2-swap local search until no swap improves (n = 1,000: 499,500 neighbours per
+    sweep).  Every accepted move is replayed through the oracle; the end point is checked to be a
+    local optimum on a sample of its neighbourhood."""
+    inst = W.mixed_1k()
+    n = inst.n
+    with kv.Scheduler(inst.s, inst.o, inst.M) as h:
+        base, _, tel0 = h.sorted_f()
+        final, tel, done, trace = h.local_search(kv.NBHD_SWAP, 5000)
+        assert done < 5000 and len(trace) == done
+        cur, cur_tel = base, tel0
+        for code, best in trace[:-1]:                              # all but the last sweep were accepted
+            cur = orc.apply_move(cur, *orc.decode_move(n, int(code)))
+            assert best < cur_tel
+            cur_tel = int(best)
+        assert trace[-1][1] >= cur_tel                             # the last sweep found nothing better
+        assert (final == cur).all() and tel == cur_tel
+        assert orc.list_schedule_rounds(inst.s, inst.o, inst.M, final)[1] == tel
+        # spot checks of accepted TELs by the oracle, spread over the run
+        cur = base
+        for k, (code, best) in enumerate(trace[:-1]):
+            cur = orc.apply_move(cur, *orc.decode_move(n, int(code)))
+            if k % 16 == 0:
+                assert orc.list_schedule_rounds(inst.s, inst.o, inst.M, cur)[1] == best
+        codes = (W.u64(8, 0, np.arange(600)) % np.uint64(n * (n - 1) // 2)).astype(np.int64)
+        assert oracle_moves(inst.s, inst.o, inst.M, final, codes).min() >= tel
+    assert tel < tel0
+
+
 def test_heavy_100k_backlog():
     """n = 100,000, o up to 4,096 (shared-memory simulator, strided snapshots), int64 TELs."""
     inst = W.heavy_100k()
