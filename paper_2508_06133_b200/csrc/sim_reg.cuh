@@ -23,6 +23,17 @@
 
 #include "common.cuh"
 
+// a + b issued as a multiply-add by one (the multiplier is read from constant memory so that it is
+// not folded away): on B200 plain integer adds, max/min, compares and selects all go through the
+// half-rate integer ALU pipe, multiply-adds through the FMA pipe, so moving the ramp adds there
+// relieves the pipe that limits this kernel.
+__constant__ int kv_const_one = 1;
+__device__ __forceinline__ int kv_add_fma_pipe(int a, int b) {
+    int r;
+    asm("mad.lo.s32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(kv_const_one), "r"(b));
+    return r;
+}
+
 // The passes over the window are specialised on a bucket (KLO, KHI] of the chunk count nch, chosen
 // by a short tree of warp-uniform branches: chunks 1 .. KLO-1 are certainly inside the window (one
 // instruction each), chunks KLO .. KHI-1 are masked by lane, and no other register is touched.
@@ -100,10 +111,10 @@ struct RegSim {
     }
     template <int KLO, int KHI>
     __device__ __forceinline__ void pass_add(int rl, int ol, int k0) {
-        if (rl >= 0 && ol > 0) R[0] += k0;
+        if (rl >= 0 && ol > 0) R[0] = kv_add_fma_pipe(R[0], k0);
 #pragma unroll
         for (int c = 1; c < KHI; ++c)
-            if (c < KLO || 32 * c < ol) R[c] += k0 + 32 * c;
+            if (c < KLO || 32 * c < ol) R[c] = kv_add_fma_pipe(R[c], k0 + 32 * c);
     }
     template <int KLO, int KHI>
     __device__ __forceinline__ int pass_need(int rl, int ol, int kadm) const {
