@@ -117,7 +117,7 @@ void free_ctx(sched_ctx* h) {
                     h->d_base_tel, h->d_counter, h->d_status, h->d_tel, h->d_best, h->d_partials, h->d_ticket,
                     h->d_keys_a, h->d_keys_b, h->d_vals_a, h->d_vals_b, h->d_prefP, h->d_prefO,
                     h->d_batch_off, h->d_num_batches, h->d_seg_off, h->d_stage, h->d_base_starts,
-                    h->d_state, h->d_sort};
+                    h->d_state, h->d_sort, h->d_k4};
     for (void* p : ptrs) if (p) cudaFree(p);
     if (h->h_pinned) cudaFreeHost(h->h_pinned);
     if (h->ev_k3_begin) cudaEventDestroy(h->ev_k3_begin);
@@ -236,7 +236,8 @@ int create_common(sched_ctx** out, int B, int n, const int32_t* s, const int32_t
 #define SETATTR(N)                                                                                         \
             e1 = cudaFuncSetAttribute(k3_eval_moves<N, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn);  \
             if (e1 == cudaSuccess) e1 = cudaFuncSetAttribute(k3_eval_moves<N, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn);  \
-            e2 = cudaFuncSetAttribute(k3_eval_orders<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn); \
+            e2 = cudaFuncSetAttribute(k3_eval_orders<N, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn); \
+            if (e2 == cudaSuccess) e2 = cudaFuncSetAttribute(k3_eval_orders<N, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn); \
             e3 = cudaFuncSetAttribute(k3_eval_policy<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn); \
             e4 = cudaFuncSetAttribute(k3_base_run<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn)
             KV_DISPATCH_SIM(h, SETATTR);
@@ -270,12 +271,33 @@ int ensure_base(sched_ctx* h) {
     return SCHED_OK;
 }
 
-int k3_grid(const sched_ctx* h, i64 count) {
+// one warp per candidate: CTAs needed for `count` candidates
+unsigned k3_grid(const sched_ctx* h, i64 count) {
     const int w = k3_warps(h);
-    i64 ctas = (count + w - 1) / w;
-    if (ctas > h->sm_count) ctas = h->sm_count;
-    if (ctas < 1) ctas = 1;
-    return (int)ctas;
+    const i64 ctas = (count + w - 1) / w;
+    return (unsigned)(ctas < 1 ? 1 : ctas);
+}
+
+// K4: launch order of `count` candidates, bucketed by first moved position (longest suffix first)
+int order_candidates(sched_ctx* h, const MoveSource& src, i64 count) {
+    const size_t need = ((size_t)h->n + 1 + 2 * (size_t)count) * sizeof(int) + 256;
+    if (h->k4_cap < need) {
+        if (h->d_k4) { cudaFree(h->d_k4); h->d_k4 = nullptr; h->k4_cap = 0; }
+        KV_CUDA(cudaMalloc(&h->d_k4, need));
+        h->k4_cap = need;
+    }
+    int* bins = (int*)h->d_k4;
+    int* first_pos = bins + h->n + 1;
+    int* launch_order = first_pos + count;
+    KV_CUDA(cudaMemsetAsync(bins, 0, ((size_t)h->n + 1) * sizeof(int), h->stream));
+    const unsigned blocks = (unsigned)((count + 255) / 256);
+    k4_first_pos_histogram<<<blocks, 256, 0, h->stream>>>(src, h->n, count, bins, first_pos);
+    KV_TRY(check_launch(h));
+    k4_scan_bins<<<1, 1024, 0, h->stream>>>(bins, h->n);
+    KV_TRY(check_launch(h));
+    k4_scatter_by_first_pos<<<blocks, 256, 0, h->stream>>>(first_pos, count, bins, launch_order);
+    KV_TRY(check_launch(h));
+    return SCHED_OK;
 }
 
 int launch_moves(sched_ctx* h, int mode, const i64* codes, i64 first, u64 seed, int iteration,
@@ -290,11 +312,12 @@ int launch_moves(sched_ctx* h, int mode, const i64* codes, i64 first, u64 seed, 
     p.n = h->n; p.L = h->L; p.M = (int)h->M; p.stride = h->snap_stride;
     p.tbl_base = h->d_tbl_base; p.table_in_smem = in_smem ? 1 : 0; p.table_bytes = tb;
     p.snap_ring = h->d_snap_ring; p.snap_hdr = h->d_snap_hdr;
-    p.mode = mode; p.codes = codes; p.first = first; p.seed = seed; p.iteration = iteration;
+    p.src.mode = mode; p.src.codes = codes; p.src.first = first; p.src.seed = seed; p.src.iteration = iteration;
     p.count = count; p.tel_out = tel_out; p.starts_out = starts_out;
     p.base_order = h->d_order; p.base_starts_pos = h->d_base_starts;
-    p.counter = h->d_counter; p.status = h->d_status;
-    KV_CUDA(cudaMemsetAsync(h->d_counter, 0, sizeof(unsigned), h->stream));
+    p.status = h->d_status;
+    KV_TRY(order_candidates(h, p.src, count));
+    p.launch_order = (const int*)h->d_k4 + h->n + 1 + count;
     KV_CUDA(cudaEventRecord(h->ev_k3_begin, h->stream));
 #define RUN(N)                                                                                    \
     if (starts_out) k3_eval_moves<N, true><<<k3_grid(h, count), k3_warps(h) * 32, smem, h->stream>>>(p);  \
@@ -426,10 +449,11 @@ int sched_eval_batch_dev(sched_handle h, int kind, int64_t count, const void* ca
         p.n = n; p.L = h->L; p.M = (int)h->M; p.tbl_id = h->d_tbl_id;
         p.table_in_smem = in_smem ? 1 : 0; p.table_bytes = tb;
         p.orders = (const int*)candidates; p.count = count; p.tel_out = (i64*)tel_out; p.starts_out = starts_out;
-        p.counter = h->d_counter; p.status = h->d_status;
-        KV_CUDA(cudaMemsetAsync(h->d_counter, 0, sizeof(unsigned), h->stream));
+        p.status = h->d_status;
         KV_CUDA(cudaEventRecord(h->ev_k3_begin, h->stream));
-#define RUN(N) k3_eval_orders<N><<<k3_grid(h, count), k3_warps(h) * 32, smem, h->stream>>>(p)
+#define RUN(N)                                                                                     \
+        if (starts_out) k3_eval_orders<N, true><<<k3_grid(h, count), k3_warps(h) * 32, smem, h->stream>>>(p);  \
+        else k3_eval_orders<N, false><<<k3_grid(h, count), k3_warps(h) * 32, smem, h->stream>>>(p)
         KV_DISPATCH_SIM(h, RUN);
 #undef RUN
         KV_TRY(check_launch(h));

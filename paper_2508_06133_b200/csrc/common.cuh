@@ -46,6 +46,8 @@ struct sched_ctx {
     void* h_pinned;          // 64 bytes of pinned host memory for small read-backs
     void* d_sort;            // grow-only scratch for sorting explicit start times
     size_t sort_cap;
+    void* d_k4;              // grow-only scratch of the launch ordering: bins[n+1], first_pos[count], order[count]
+    size_t k4_cap;
 
     // snapshots of the base run
     int snap_stride, snap_count;

@@ -3,9 +3,10 @@
 //   k3_gather_table   (s, o) of the request at every position of the base order.
 //   k3_base_run       one warp list-schedules the base order and stores the simulator state in
 //                     front of every `stride`-th position (snapshots) plus the start of every position.
-//   k3_eval_moves     persistent CTAs, one warp per candidate; the candidate is a move applied to
-//                     the base order (K4: code -> (type, i, j) -> position map, never materialised);
-//                     simulation resumes from the last snapshot at or before the first moved position.
+//   k3_eval_moves     one warp per candidate; the candidate is a move applied to the base order
+//                     (K4: index -> (type, i, j) -> position map, never materialised; launch order
+//                     bucketed by first moved position); simulation resumes from the last snapshot
+//                     at or before the first moved position.
 //   k3_eval_orders    explicit permutations, simulated from t = 0.
 //   k3_eval_policy    one single-warp CTA per (instance, policy) pair: sort, optional prefix-F
 //                     batching, simulation -- all in shared memory.
@@ -18,6 +19,7 @@
 
 #include "common.cuh"
 #include "k2_fmetric.cuh"
+#include "k4_moves.cuh"
 #include "sim.cuh"
 #include "sim_reg.cuh"
 
@@ -132,20 +134,19 @@ struct MoveEvalParams {
     unsigned table_bytes;              // multiple of 16
     const int* snap_ring;
     const SnapHeader* snap_hdr;
-    int mode;
-    const i64* codes;
-    i64 first;
-    u64 seed;
-    int iteration;
+    MoveSource src;
     i64 count;
+    const int* launch_order;           // candidate index of every launch slot (K4)
     i64* tel_out;
     int* starts_out;                   // nullable [count][n], by request id
     const int* base_order;
     const int* base_starts_pos;
-    unsigned int* counter;
     int* status;
 };
 
+// One warp per candidate, no loop over candidates (a persistent loop around the simulator costs
+// ~15 % more instructions per admission with this compiler): warp w of CTA b takes launch slot
+// 32 b + w, whose candidate K4 chose so that the warps of a CTA have nearly equal work.
 template <class SIM, bool kStarts>
 __global__ void __launch_bounds__(SIM::kWarps * 32, 1)
 k3_eval_moves(const MoveEvalParams p) {
@@ -161,44 +162,37 @@ k3_eval_moves(const MoveEvalParams p) {
         ring_off = (p.table_bytes + 127) & ~(size_t)127;
     }
     const int n = p.n, L = p.L, M = p.M;
+    const i64 slot = (i64)blockIdx.x * (blockDim.x >> 5) + warp;
+    if (slot >= p.count) return;
+    const i64 c = p.launch_order[slot];
     SIM sim;
     sim.attach((int*)(smem_raw + ring_off) + (size_t)warp * L, L);
-
-    for (;;) {
-        unsigned c32 = 0;
-        if (lane == 0) c32 = atomicAdd(p.counter, 1u);
-        const i64 c = (i64)__shfl_sync(KV_FULL, c32, 0);
-        if (c >= p.count) break;
-        Move mv;
-        if (p.mode == 0) mv = kv_decode_move(n, p.codes[c]);
-        else if (p.mode == 1) mv = kv_decode_move(n, p.first + c);
-        else mv = kv_sample_move(n, p.seed, p.iteration, p.first + c);
-        const int first_pos = min(mv.i, mv.j);
-        const int idx = first_pos / p.stride;
-        const int q_start = idx * p.stride;
-        // restore the base run's state in front of q_start
-        sim.load(p.snap_ring + (size_t)idx * L, p.snap_hdr[idx], lane);
-        int* starts = kStarts ? p.starts_out + (size_t)c * n : nullptr;
-        if (kStarts)
-            for (int q = lane; q < q_start; q += 32) starts[p.base_order[q]] = p.base_starts_pos[q];
-        for (int q0 = q_start; q0 < n; q0 += 32) {
-            const int qq = q0 + lane;
-            int2 so = make_int2(1, 1);
-            int id = 0;
-            if (qq < n) {
-                const int bp = kv_map_pos(mv, qq);
-                so = tbl[bp];
-                if (kStarts) id = p.base_order[bp];
-            }
-            const int cnt = min(32, n - q0);
-            for (int k = 0; k < cnt; ++k) {
-                const int s = __shfl_sync(KV_FULL, so.x, k), o = __shfl_sync(KV_FULL, so.y, k);
-                const int pstart = sim.admit(s, o, M, lane, p.status);
-                if (kStarts && lane == k) starts[id] = pstart;
-            }
+    const Move mv = k4_move_of(p.src, n, c);
+    const int first_pos = min(mv.i, mv.j);
+    const int idx = first_pos / p.stride;
+    const int q_start = idx * p.stride;
+    // restore the base run's state in front of q_start
+    sim.load(p.snap_ring + (size_t)idx * L, p.snap_hdr[idx], lane);
+    int* starts = kStarts ? p.starts_out + (size_t)c * n : nullptr;
+    if (kStarts)
+        for (int q = lane; q < q_start; q += 32) starts[p.base_order[q]] = p.base_starts_pos[q];
+    for (int q0 = q_start; q0 < n; q0 += 32) {
+        const int qq = q0 + lane;
+        int2 so = make_int2(1, 1);
+        int id = 0;
+        if (qq < n) {
+            const int bp = kv_map_pos(mv, qq);
+            so = tbl[bp];
+            if (kStarts) id = p.base_order[bp];
         }
-        if (lane == 0) p.tel_out[c] = sim.total();
+        const int cnt = min(32, n - q0);
+        for (int k = 0; k < cnt; ++k) {
+            const int s = __shfl_sync(KV_FULL, so.x, k), o = __shfl_sync(KV_FULL, so.y, k);
+            const int pstart = sim.admit(s, o, M, lane, p.status);
+            if (kStarts && lane == k) starts[id] = pstart;
+        }
     }
+    if (lane == 0) p.tel_out[c] = sim.total();
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -213,11 +207,10 @@ struct OrderEvalParams {
     i64 count;
     i64* tel_out;
     int* starts_out;
-    unsigned int* counter;
     int* status;
 };
 
-template <class SIM>
+template <class SIM, bool kStarts>
 __global__ void __launch_bounds__(SIM::kWarps * 32, 1)
 k3_eval_orders(const OrderEvalParams p) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -232,30 +225,26 @@ k3_eval_orders(const OrderEvalParams p) {
         ring_off = (p.table_bytes + 127) & ~(size_t)127;
     }
     const int n = p.n, L = p.L, M = p.M;
+    const i64 c = (i64)blockIdx.x * (blockDim.x >> 5) + warp;      // every order has the same length
+    if (c >= p.count) return;
     SIM sim;
     sim.attach((int*)(smem_raw + ring_off) + (size_t)warp * L, L);
-    for (;;) {
-        unsigned c32 = 0;
-        if (lane == 0) c32 = atomicAdd(p.counter, 1u);
-        const i64 c = (i64)__shfl_sync(KV_FULL, c32, 0);
-        if (c >= p.count) break;
-        const int* ord = p.orders + (size_t)c * n;
-        int* starts = p.starts_out ? p.starts_out + (size_t)c * n : nullptr;
-        sim.reset(lane);
-        for (int q0 = 0; q0 < n; q0 += 32) {
-            const int qq = q0 + lane;
-            int2 so = make_int2(1, 1);
-            int id = 0;
-            if (qq < n) { id = ord[qq]; so = tbl[id]; }
-            const int cnt = min(32, n - q0);
-            for (int k = 0; k < cnt; ++k) {
-                const int s = __shfl_sync(KV_FULL, so.x, k), o = __shfl_sync(KV_FULL, so.y, k);
-                const int pstart = sim.admit(s, o, M, lane, p.status);
-                if (starts && lane == k) starts[id] = pstart;
-            }
+    const int* ord = p.orders + (size_t)c * n;
+    int* starts = kStarts ? p.starts_out + (size_t)c * n : nullptr;
+    sim.reset(lane);
+    for (int q0 = 0; q0 < n; q0 += 32) {
+        const int qq = q0 + lane;
+        int2 so = make_int2(1, 1);
+        int id = 0;
+        if (qq < n) { id = ord[qq]; so = tbl[id]; }
+        const int cnt = min(32, n - q0);
+        for (int k = 0; k < cnt; ++k) {
+            const int s = __shfl_sync(KV_FULL, so.x, k), o = __shfl_sync(KV_FULL, so.y, k);
+            const int pstart = sim.admit(s, o, M, lane, p.status);
+            if (kStarts && lane == k) starts[id] = pstart;
         }
-        if (lane == 0) p.tel_out[c] = sim.total();
     }
+    if (lane == 0) p.tel_out[c] = sim.total();
 }
 
 // ------------------------------------------------------------------------------------------------
