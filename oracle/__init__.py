@@ -195,3 +195,27 @@ def bruteforce_best_order(s, o, M):
     order = np.zeros(len(s), dtype=np.int32)
     v = lib().orc_bruteforce_best_order(len(s), _p(s), _p(o), C.c_longlong(M), _p(order))
     return v, order
+
+
+def local_swap_batch(ids, s, o, M):
+    """Algorithm 4 on the request set ``ids``.  Returns (X in walking order, accepted swaps)."""
+    s, o, ids = _i32(s), _i32(o), _i32(ids)
+    chosen = np.zeros(len(ids), dtype=np.int32)
+    sw = C.c_longlong(0)
+    c = lib().orc_local_swap_batch(len(ids), _p(ids), _p(s), _p(o), C.c_longlong(M), _p(chosen), C.byref(sw))
+    if c < 0:
+        raise ValueError("a request exceeds M")
+    return chosen[:c].copy(), sw.value
+
+
+def sorted_f_local_swap(s, o, M):
+    """Sorted-F with Algorithm 4 as Phase-1 solver.  Returns (order, batch offsets, accepted swaps)."""
+    s, o = _i32(s), _i32(o)
+    n = len(s)
+    order = np.zeros(n, dtype=np.int32)
+    offs = np.zeros(n + 1, dtype=np.int32)
+    sw = C.c_longlong(0)
+    nb = lib().orc_sorted_f_local_swap(n, _p(s), _p(o), C.c_longlong(M), _p(order), _p(offs), C.byref(sw))
+    if nb < 0:
+        raise ValueError("a request exceeds M")
+    return order, offs[:nb + 1].copy(), sw.value

@@ -486,4 +486,85 @@ i64 orc_bruteforce_best_order(int n, const int* s, const int* o, i64 M, int* bes
     return best;
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// O10. Algorithm 4 (Local Swap Search), as printed: one batch out of the request set `ids`.
+//      Sort by ascending s+o (ties: lower index); first-fit fill in that order; then repeat: walk
+//      r_out over X and r_in over the requests outside X, take the FIRST pair that keeps
+//      sum(s+o) <= M and lowers F (|X| is fixed, so F drops iff o_in < o_out), swap, start over;
+//      stop when no pair qualifies.  Orders the listing leaves open: X is walked in insertion order
+//      with a swapped-in request taking the place of the one it replaces; the outside requests are
+//      walked in the sorted order.
+// Writes X (in its walking order) and returns |X|.  swaps_out (nullable) counts accepted swaps.
+// ---------------------------------------------------------------------------------------------
+int orc_local_swap_batch(int m, const int* ids, const int* s, const int* o, i64 M, int* chosen, i64* swaps_out) {
+    std::vector<int> I(ids, ids + m);
+    std::stable_sort(I.begin(), I.end(), [&](int a, int b) {
+        int ta = s[a] + o[a], tb = s[b] + o[b];
+        if (ta != tb) return ta < tb;
+        return a < b;
+    });
+    std::vector<int> X;
+    std::vector<char> inX(m, 0);                     // by position in I
+    std::vector<int> posX;                           // position in I of every member of X
+    i64 mem = 0, swaps = 0;
+    for (int p = 0; p < m; ++p) {
+        int r = I[p];
+        if (mem + s[r] + o[r] <= M) { X.push_back(r); posX.push_back(p); inX[p] = 1; mem += s[r] + o[r]; }
+    }
+    if (X.empty()) return -1;
+    bool improved = true;
+    while (improved) {
+        improved = false;
+        i64 sum_o = 0;
+        for (int r : X) sum_o += o[r];
+        for (size_t k = 0; k < X.size() && !improved; ++k) {
+            int rout = X[k];
+            for (int p = 0; p < m; ++p) {
+                if (inX[p]) continue;
+                int rin = I[p];
+                i64 dm = (i64)(s[rin] + o[rin]) - (s[rout] + o[rout]);
+                if (mem + dm > M) continue;
+                i64 d_o = (i64)o[rin] - o[rout];
+                // newF < currentF with the same |X|:  (sum_o + d_o) / k^2 < sum_o / k^2
+                if (sum_o + d_o < sum_o) {
+                    inX[posX[k]] = 0; inX[p] = 1; posX[k] = p; X[k] = rin;
+                    mem += dm; improved = true; ++swaps;
+                    break;
+                }
+            }
+        }
+    }
+    for (size_t k = 0; k < X.size(); ++k) chosen[k] = X[k];
+    if (swaps_out) *swaps_out = swaps;
+    return (int)X.size();
+}
+
+// Sorted-F with Algorithm 4 as the Phase-1 solver (what Section 7 calls Sorted-F with Local Swap
+// Search): repeat { X = Algorithm 4 on the remaining requests; sort X by (o, index); append }.
+int orc_sorted_f_local_swap(int n, const int* s, const int* o, i64 M, int* order, int* batch_offsets, i64* swaps_out) {
+    std::vector<int> rem(n);
+    std::iota(rem.begin(), rem.end(), 0);
+    std::vector<int> chosen(n);
+    int pos = 0, nb = 0;
+    i64 swaps = 0;
+    batch_offsets[0] = 0;
+    while (!rem.empty()) {
+        i64 sw = 0;
+        int c = orc_local_swap_batch((int)rem.size(), rem.data(), s, o, M, chosen.data(), &sw);
+        if (c <= 0) return -1;
+        swaps += sw;
+        std::vector<int> X(chosen.begin(), chosen.begin() + c);
+        std::sort(X.begin(), X.end(), [&](int a, int b) { if (o[a] != o[b]) return o[a] < o[b]; return a < b; });
+        std::vector<char> gone(n, 0);
+        for (int x : X) { order[pos++] = x; gone[x] = 1; }
+        batch_offsets[++nb] = pos;
+        std::vector<int> rest;
+        for (int r : rem) if (!gone[r]) rest.push_back(r);
+        rem.swap(rest);
+    }
+    if (swaps_out) *swaps_out = swaps;
+    return nb;
+}
+
 }  // extern "C"

@@ -409,3 +409,56 @@ def test_workloads_are_deterministic_and_shaped():
     assert (big.s.astype(np.int64) + big.o).sum() > 20 * big.M          # overloaded regime
     t = W.tiny()
     assert t.n == 16 and t.s.min() >= 1 and t.s.max() <= 32 and t.o.min() >= 1 and t.o.max() <= 32
+
+
+# ----------------------------------------------------------------------------- Algorithm 4 (Local Swap Search)
+def test_local_swap_worked_by_hand():
+    # A(1,5) B(2,5) C(5,3) D(8,1) E(9,1); sizes 6,7,8,9,10; M = 14.
+    # First fit: A, B (mem 13).  out=A: C,D,E all overflow.  out=B: C fits exactly (14) and has the
+    # smaller o -> X = [A, C].  Restart: nothing outside is both smaller in o and fits -> stop.
+    s, o = np.array([1, 2, 5, 8, 9], dtype=np.int32), np.array([5, 5, 3, 1, 1], dtype=np.int32)
+    X, swaps = orc.local_swap_batch(np.arange(5), s, o, 14)
+    assert X.tolist() == [0, 2] and swaps == 1
+    # equal sizes: the walk is out-major, in-minor and restarts after every swap.
+    # P(4,6) Q(4,6) R(6,4) S(8,2), all of size 10, M = 20: P->R, then R->S, then Q->R.
+    s, o = np.array([4, 4, 6, 8], dtype=np.int32), np.array([6, 6, 4, 2], dtype=np.int32)
+    X, swaps = orc.local_swap_batch(np.arange(4), s, o, 20)
+    assert X.tolist() == [3, 2] and swaps == 3
+
+
+def test_local_swap_example1_and_properties(golden):
+    s = np.array([63] + [1] * 21, dtype=np.int32)
+    o = np.array([1] + [2] * 21, dtype=np.int32)
+    order, offs, swaps = orc.sorted_f_local_swap(s, o, golden["example1_M"])
+    assert offs.tolist() == [0, 21, 22] and order[-1] == 0 and swaps == 0
+    assert orc.list_schedule_alg1(s, o, 64, order)[1] == golden["example1_tel_sortedf"]
+    rng = np.random.default_rng(404)
+    for trial in range(150):
+        n = int(rng.integers(1, 40))
+        M = int(rng.integers(10, 120))
+        s, o = random_instance(rng, n, M, M // 2, M // 2)
+        ids = np.arange(n)
+        X, swaps = orc.local_swap_batch(ids, s, o, M)
+        T = s.astype(np.int64) + o
+        mem = int(T[X].sum())
+        assert len(set(X.tolist())) == len(X) and mem <= M
+        # the batch size is the first-fit size: the longest prefix by ascending s+o that fits
+        by_size = sorted(range(n), key=lambda i: (T[i], i))
+        k0, acc = 0, 0
+        for i in by_size:
+            if acc + T[i] <= M:
+                acc += T[i]; k0 += 1
+        assert len(X) == k0
+        # local optimum by the definition of Section 5.2: no swap keeps memory and lowers F
+        outside = [i for i in range(n) if i not in set(X.tolist())]
+        for a in X:
+            for b in outside:
+                assert not (mem + T[b] - T[a] <= M and o[b] < o[a])
+        # never worse than where it started
+        assert int(o[X].sum()) <= int(o[by_size[:k0]].sum())
+        assert (swaps == 0) == (sorted(X.tolist()) == sorted(by_size[:k0]))
+        order, offs, _ = orc.sorted_f_local_swap(s, o, M)
+        assert sorted(order.tolist()) == list(range(n)) and offs[0] == 0 and offs[-1] == n
+        for a, b in zip(offs[:-1], offs[1:]):
+            assert (np.diff(o[order[a:b]]) >= 0).all() and int(T[order[a:b]].sum()) <= M
+        assert order[:offs[1]].tolist() == sorted(X.tolist(), key=lambda i: (o[i], i))
