@@ -140,6 +140,21 @@ int sched_sorted_f(sched_handle h, int32_t* order_out, int32_t* batch_offsets_ou
 int sched_sorted_f_dev(sched_handle h, int32_t* order_out, int32_t* batch_offsets_out,
                        int32_t* num_batches_out, int64_t* tel_out);
 
+/* Sorted-F with Algorithm 4 (Local Swap Search, Section 5.2 and Appendix D) as the Phase-1 solver --
+ * the variant the paper's experiments use at n = 2000.  Repeat on the requests not yet placed:
+ * sort by ascending s+o (ties: lower index); first-fit fill up to sum(s+o) <= M; then, walking
+ * r_out over the batch (insertion order; a swapped-in request takes the replaced one's place) and
+ * r_in over the outside requests (sorted order), swap the first pair that keeps sum(s+o) <= M and
+ * lowers F (same batch size, so iff o_in < o_out) and start the walk over, until no pair
+ * qualifies; sort the batch by (o, index) and append it.  Outputs and side effects as
+ * sched_sorted_f(): the order becomes the handle's base order.  Single-instance handles only. */
+int sched_sorted_f_local_swap(sched_handle h, int32_t* order_out, int32_t* batch_offsets_out,
+                              int32_t* num_batches_out, int64_t* tel_out);
+
+/* Same, results left on the device; asynchronous (see sched_sorted_f_dev). */
+int sched_sorted_f_local_swap_dev(sched_handle h, int32_t* order_out, int32_t* batch_offsets_out,
+                                  int32_t* num_batches_out, int64_t* tel_out);
+
 /* Order-level local search from order_inout (NULL: from the handle's base order).  Each iteration
  * evaluates the whole neighbourhood with Algorithm 1 Phase 2, takes the best (TEL, code) pair --
  * lowest code among equal TELs -- and accepts it iff its TEL is strictly below the current one

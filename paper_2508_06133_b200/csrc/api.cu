@@ -11,6 +11,7 @@
 #include "common.cuh"
 #include "k1_sort.cuh"
 #include "k2_fmetric.cuh"
+#include "k2_local_swap.cuh"
 #include "k3_eval.cuh"
 #include "k5_argmin.cuh"
 
@@ -117,7 +118,7 @@ void free_ctx(sched_ctx* h) {
                     h->d_base_tel, h->d_counter, h->d_status, h->d_tel, h->d_best, h->d_partials, h->d_ticket,
                     h->d_keys_a, h->d_keys_b, h->d_vals_a, h->d_vals_b, h->d_prefP, h->d_prefO,
                     h->d_batch_off, h->d_num_batches, h->d_seg_off, h->d_stage, h->d_base_starts,
-                    h->d_state, h->d_sort, h->d_k4};
+                    h->d_state, h->d_sort, h->d_k4, h->d_ls};
     for (void* p : ptrs) if (p) cudaFree(p);
     if (h->h_pinned) cudaFreeHost(h->h_pinned);
     if (h->ev_k3_begin) cudaEventDestroy(h->ev_k3_begin);
@@ -573,21 +574,37 @@ int sched_sweep_dev(sched_handle h, int sampled, uint64_t seed, int32_t iteratio
     return SCHED_OK;
 }
 
-int sched_sorted_f_dev(sched_handle h, int32_t* order_out, int32_t* batch_offsets_out,
-                       int32_t* num_batches_out, int64_t* tel_out) {
+static int sorted_f_common_dev(sched_handle h, int solver, int32_t* order_out, int32_t* batch_offsets_out,
+                               int32_t* num_batches_out, int64_t* tel_out) {
     KV_ENTER(h);
     if (h->batch_handle) return SCHED_E_INVAL;
     const int n = h->n;
     cudaStream_t st = h->stream;
-    // S1: ascending (s+o, o, index)
-    k1_keys_total_size<<<(n + 255) / 256, 256, 0, st>>>(h->d_s, h->d_o, n, h->d_keys_a, h->d_vals_a, SCHED_POLICY_SORTED_F);
-    KV_TRY(check_launch(h));
-    k1_radix_sort_segments<<<1, K1_THREADS, 0, st>>>(h->d_keys_a, h->d_vals_a, h->d_keys_b, h->d_vals_b, h->d_seg_off, nullptr, 1,
-                                                      key_byte_mask(bits_of((u64)h->omax), bits_of((u64)h->M)));
-    KV_TRY(check_launch(h));
-    // S2: prefix sums + F-metric batch boundaries
-    k2_prefix_f<<<1, 1024, 0, st>>>(h->d_s, h->d_o, h->d_vals_a, n, h->M, h->d_prefP, h->d_prefO, h->d_batch_off, h->d_num_batches);
-    KV_TRY(check_launch(h));
+    if (solver == 0) {
+        // S1: ascending (s+o, o, index)
+        k1_keys_total_size<<<(n + 255) / 256, 256, 0, st>>>(h->d_s, h->d_o, n, h->d_keys_a, h->d_vals_a, SCHED_POLICY_SORTED_F);
+        KV_TRY(check_launch(h));
+        k1_radix_sort_segments<<<1, K1_THREADS, 0, st>>>(h->d_keys_a, h->d_vals_a, h->d_keys_b, h->d_vals_b, h->d_seg_off, nullptr, 1,
+                                                          key_byte_mask(bits_of((u64)h->omax), bits_of((u64)h->M)));
+        KV_TRY(check_launch(h));
+        // S2: prefix sums + F-metric batch boundaries
+        k2_prefix_f<<<1, 1024, 0, st>>>(h->d_s, h->d_o, h->d_vals_a, n, h->M, h->d_prefP, h->d_prefO, h->d_batch_off, h->d_num_batches);
+        KV_TRY(check_launch(h));
+    } else {
+        // Algorithm 4: ascending (s+o, index), then first fit + improving swaps, batch after batch
+        if (!h->d_ls) KV_TRY(dev_alloc(&h->d_ls, 7 * (size_t)n));
+        k1_keys_total_size<<<(n + 255) / 256, 256, 0, st>>>(h->d_s, h->d_o, n, h->d_keys_a, h->d_vals_a, SCHED_POLICY_TOTAL_SIZE);
+        KV_TRY(check_launch(h));
+        k1_radix_sort_segments<<<1, K1_THREADS, 0, st>>>(h->d_keys_a, h->d_vals_a, h->d_keys_b, h->d_vals_b, h->d_seg_off, nullptr, 1,
+                                                          key_byte_mask(0, bits_of((u64)h->M)));
+        KV_TRY(check_launch(h));
+        int* ls = h->d_ls;
+        k2_local_swap<<<1, K2L_THREADS, 0, st>>>(h->d_s, h->d_o, h->d_vals_a, n, h->M, ls, ls + n, ls + 2 * (size_t)n,
+                                                 ls + 3 * (size_t)n, ls + 4 * (size_t)n, ls + 5 * (size_t)n, ls + 6 * (size_t)n,
+                                                 h->d_vals_b, h->d_batch_off, h->d_num_batches, h->d_status);
+        KV_TRY(check_launch(h));
+        KV_CUDA(cudaMemcpyAsync(h->d_vals_a, h->d_vals_b, (size_t)n * sizeof(int), cudaMemcpyDeviceToDevice, st));
+    }
     // each batch by ascending (o, index)
     k1_keys_output_then_id<<<(n + 255) / 256, 256, 0, st>>>(h->d_o, h->d_vals_a, n, h->d_keys_a, h->d_vals_a);
     KV_TRY(check_launch(h));
@@ -605,10 +622,10 @@ int sched_sorted_f_dev(sched_handle h, int32_t* order_out, int32_t* batch_offset
     return SCHED_OK;
 }
 
-int sched_sorted_f(sched_handle h, int32_t* order_out, int32_t* batch_offsets_out,
-                   int32_t* num_batches_out, int64_t* tel_out) {
+static int sorted_f_common_host(sched_handle h, int solver, int32_t* order_out, int32_t* batch_offsets_out,
+                                int32_t* num_batches_out, int64_t* tel_out) {
     KV_ENTER(h);
-    KV_TRY(sched_sorted_f_dev(h, nullptr, nullptr, nullptr, nullptr));
+    KV_TRY(sorted_f_common_dev(h, solver, nullptr, nullptr, nullptr, nullptr));
     const int n = h->n;
     cudaStream_t st = h->stream;
     int nb = 0;
@@ -621,6 +638,26 @@ int sched_sorted_f(sched_handle h, int32_t* order_out, int32_t* batch_offsets_ou
         KV_CUDA(cudaMemcpyAsync(batch_offsets_out, h->d_batch_off, (size_t)(nb + 1) * sizeof(int), cudaMemcpyDeviceToHost, st));
     }
     return read_status(h);
+}
+
+int sched_sorted_f_dev(sched_handle h, int32_t* order_out, int32_t* batch_offsets_out,
+                       int32_t* num_batches_out, int64_t* tel_out) {
+    return sorted_f_common_dev(h, 0, order_out, batch_offsets_out, num_batches_out, tel_out);
+}
+
+int sched_sorted_f_local_swap_dev(sched_handle h, int32_t* order_out, int32_t* batch_offsets_out,
+                                  int32_t* num_batches_out, int64_t* tel_out) {
+    return sorted_f_common_dev(h, 1, order_out, batch_offsets_out, num_batches_out, tel_out);
+}
+
+int sched_sorted_f_local_swap(sched_handle h, int32_t* order_out, int32_t* batch_offsets_out,
+                              int32_t* num_batches_out, int64_t* tel_out) {
+    return sorted_f_common_host(h, 1, order_out, batch_offsets_out, num_batches_out, tel_out);
+}
+
+int sched_sorted_f(sched_handle h, int32_t* order_out, int32_t* batch_offsets_out,
+                   int32_t* num_batches_out, int64_t* tel_out) {
+    return sorted_f_common_host(h, 0, order_out, batch_offsets_out, num_batches_out, tel_out);
 }
 
 int sched_local_search(sched_handle h, int neighbourhood, int32_t iters, uint64_t seed,

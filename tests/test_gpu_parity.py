@@ -184,6 +184,30 @@ def test_sorted_f_example1(golden):
     assert offs.tolist() == [0, 21, 22] and order[-1] == 0 and tel == golden["example1_tel_sortedf"]
 
 
+def test_sorted_f_local_swap_matches_oracle():
+    """Sorted-F with Algorithm 4 (Local Swap Search) as Phase-1 solver: batches, order and TEL."""
+    rng = np.random.default_rng(44)
+    cases = [W.tiny(), W.mixed_1k(), W.paper_scale(), W.mixed_10k()]
+    for trial in range(40):
+        n = int(rng.integers(1, 300))
+        M = int(rng.integers(10, 1500))
+        s, o = rand_instance(rng, n, M, M // 2, max(1, M // 3))
+        cases.append(W.Instance("rand", s, o, M))
+    cases.append(W.Instance("ties", np.array([4, 4, 6, 8] * 30, dtype=np.int32), np.array([6, 6, 4, 2] * 30, dtype=np.int32), 50))
+    cases.append(W.Instance("ex1", np.array([63] + [1] * 21, dtype=np.int32), np.array([1] + [2] * 21, dtype=np.int32), 64))
+    total_swaps = 0
+    for inst in cases:
+        with kv.Scheduler(inst.s, inst.o, inst.M) as h:
+            order, offs, tel = h.sorted_f_local_swap()
+            assert (h.get_base_order() == order).all()
+        r_order, r_offs, swaps = orc.sorted_f_local_swap(inst.s, inst.o, inst.M)
+        total_swaps += swaps
+        assert (offs == r_offs).all(), inst.name
+        assert (order == r_order).all(), inst.name
+        assert tel == orc.list_schedule_rounds(inst.s, inst.o, inst.M, r_order)[1]
+    assert total_swaps > 1000                                   # the improvement loop really ran
+
+
 # ------------------------------------------------------------------------------------ POLICY
 def test_policy_sweep_small_batch():
     s, o, M = W.policy_sweep(num_instances=24, n_each=256)
