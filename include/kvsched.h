@@ -155,6 +155,16 @@ int sched_sorted_f_local_swap(sched_handle h, int32_t* order_out, int32_t* batch
 int sched_sorted_f_local_swap_dev(sched_handle h, int32_t* order_out, int32_t* batch_offsets_out,
                                   int32_t* num_batches_out, int64_t* tel_out);
 
+/* Sorted-F with Algorithm 2 (exact dynamic programme, Section 5.1 and Appendix D) as the Phase-1
+ * solver: repeat on the requests not yet placed { dp[k][m] = min sum of o over k-subsets whose
+ * sum(s+o) is exactly m <= M, requests taken in ascending index, a cell replaced only by a strictly
+ * smaller value; the batch is the cell minimising dp/k^2, ties to the larger k (Section 3), then the
+ * smaller m, and its members are the listing's path set; sort it by (o, index); append }.
+ * Meant for small instances (the paper recommends n <= 100): SCHED_E_UNSUPPORTED if n > 128 or
+ * (n+1)*(M+1) > 2^26.  Host pointers; outputs and side effects as sched_sorted_f(). */
+int sched_sorted_f_dp(sched_handle h, int32_t* order_out, int32_t* batch_offsets_out,
+                      int32_t* num_batches_out, int64_t* tel_out);
+
 /* Order-level local search from order_inout (NULL: from the handle's base order).  Each iteration
  * evaluates the whole neighbourhood with Algorithm 1 Phase 2, takes the best (TEL, code) pair --
  * lowest code among equal TELs -- and accepts it iff its TEL is strictly below the current one

@@ -12,6 +12,7 @@
 #include "k1_sort.cuh"
 #include "k2_fmetric.cuh"
 #include "k2_local_swap.cuh"
+#include "k2_dp.cuh"
 #include "k3_eval.cuh"
 #include "k5_argmin.cuh"
 
@@ -574,6 +575,8 @@ int sched_sweep_dev(sched_handle h, int sampled, uint64_t seed, int32_t iteratio
     return SCHED_OK;
 }
 
+static int phase1_dp(sched_handle h);
+
 static int sorted_f_common_dev(sched_handle h, int solver, int32_t* order_out, int32_t* batch_offsets_out,
                                int32_t* num_batches_out, int64_t* tel_out) {
     KV_ENTER(h);
@@ -590,6 +593,8 @@ static int sorted_f_common_dev(sched_handle h, int solver, int32_t* order_out, i
         // S2: prefix sums + F-metric batch boundaries
         k2_prefix_f<<<1, 1024, 0, st>>>(h->d_s, h->d_o, h->d_vals_a, n, h->M, h->d_prefP, h->d_prefO, h->d_batch_off, h->d_num_batches);
         KV_TRY(check_launch(h));
+    } else if (solver == 2) {
+        KV_TRY(phase1_dp(h));
     } else {
         // Algorithm 4: ascending (s+o, index), then first fit + improving swaps, batch after batch
         if (!h->d_ls) KV_TRY(dev_alloc(&h->d_ls, 7 * (size_t)n));
@@ -640,6 +645,69 @@ static int sorted_f_common_host(sched_handle h, int solver, int32_t* order_out, 
     return read_status(h);
 }
 
+// Algorithm 2 batch after batch; leaves the batches (members in ascending index) in d_vals_a and the
+// boundaries in d_batch_off / d_num_batches.  Synchronises once per batch (n <= 128 batches).
+static int phase1_dp(sched_handle h) {
+    const int n = h->n;
+    if (n > 128) return SCHED_E_UNSUPPORTED;
+    const int W = (int)h->M + 1, words = (W + 31) / 32;
+    const i64 cells_max = (i64)(n + 1) * W;
+    if (cells_max > (1ll << 26)) return SCHED_E_UNSUPPORTED;
+    cudaStream_t st = h->stream;
+    int *dpA = nullptr, *dpB = nullptr, *small = nullptr;
+    unsigned* took = nullptr;
+    int rc = SCHED_OK;
+    do {
+        if ((rc = dev_alloc(&dpA, (size_t)cells_max)) != SCHED_OK) break;
+        if ((rc = dev_alloc(&dpB, (size_t)cells_max)) != SCHED_OK) break;
+        if ((rc = dev_alloc(&took, (size_t)n * (n + 1) * words)) != SCHED_OK) break;
+        if ((rc = dev_alloc(&small, 8)) != SCHED_OK) break;            // {pick k, m, v, -, nr, nb, done, -}
+        int init[8] = {0, 0, 0, 0, n, 0, 0, 0};
+        int zero = 0;
+#define DP_CUDA(call) if ((call) != cudaSuccess) { rc = kv_cuda_fail(cudaGetLastError(), #call); break; }
+        DP_CUDA(cudaMemcpyAsync(small, init, sizeof(init), cudaMemcpyHostToDevice, st));
+        DP_CUDA(cudaMemcpyAsync(h->d_batch_off, &zero, sizeof(int), cudaMemcpyHostToDevice, st));
+        k3_iota<<<(n + 255) / 256, 256, 0, st>>>(h->d_vals_b, n);       // remaining list, ascending index
+        if ((rc = check_launch(h)) != SCHED_OK) break;
+        int nr = n;
+        int* hp = (int*)h->h_pinned;
+        while (nr > 0 && rc == SCHED_OK) {
+            const int rows = nr + 1;
+            const i64 cells = (i64)rows * W;
+            k2d_init<<<(unsigned)((cells + 255) / 256), 256, 0, st>>>(dpA, cells);
+            if ((rc = check_launch(h)) != SCHED_OK) break;
+            int *cur = dpA, *nxt = dpB;
+            const i64 threads = (i64)rows * words;
+            for (int a = 0; a < nr; ++a) {
+                k2d_step<<<(unsigned)((threads + 127) / 128), 128, 0, st>>>(cur, nxt, took + (size_t)a * rows * words, rows, W, words,
+                                                                             h->d_s, h->d_o, h->d_vals_b, a);
+                if ((rc = check_launch(h)) != SCHED_OK) break;
+                int* tmp = cur; cur = nxt; nxt = tmp;
+            }
+            if (rc != SCHED_OK) break;
+            k2d_select<<<1, 1024, 0, st>>>(cur, rows, W, small);
+            if ((rc = check_launch(h)) != SCHED_OK) break;
+            k2d_apply<<<1, 128, 0, st>>>(h->d_s, h->d_o, took, W, words, rows, small, h->d_vals_b, small + 4,
+                                         h->d_vals_a, h->d_batch_off, small + 5, small + 6);
+            if ((rc = check_launch(h)) != SCHED_OK) break;
+            DP_CUDA(cudaMemcpyAsync(hp, small + 4, sizeof(int), cudaMemcpyDeviceToHost, st));
+            DP_CUDA(cudaStreamSynchronize(st));
+            if (*hp >= nr) { rc = SCHED_E_INTERNAL; break; }            // every batch places at least one request
+            nr = *hp;
+        }
+        if (rc != SCHED_OK) break;
+        DP_CUDA(cudaMemcpyAsync(h->d_num_batches, small + 5, sizeof(int), cudaMemcpyDeviceToDevice, st));
+        DP_CUDA(cudaStreamSynchronize(st));
+#undef DP_CUDA
+    } while (0);
+    cudaStreamSynchronize(st);
+    if (dpA) cudaFree(dpA);
+    if (dpB) cudaFree(dpB);
+    if (took) cudaFree(took);
+    if (small) cudaFree(small);
+    return rc;
+}
+
 int sched_sorted_f_dev(sched_handle h, int32_t* order_out, int32_t* batch_offsets_out,
                        int32_t* num_batches_out, int64_t* tel_out) {
     return sorted_f_common_dev(h, 0, order_out, batch_offsets_out, num_batches_out, tel_out);
@@ -653,6 +721,11 @@ int sched_sorted_f_local_swap_dev(sched_handle h, int32_t* order_out, int32_t* b
 int sched_sorted_f_local_swap(sched_handle h, int32_t* order_out, int32_t* batch_offsets_out,
                               int32_t* num_batches_out, int64_t* tel_out) {
     return sorted_f_common_host(h, 1, order_out, batch_offsets_out, num_batches_out, tel_out);
+}
+
+int sched_sorted_f_dp(sched_handle h, int32_t* order_out, int32_t* batch_offsets_out,
+                      int32_t* num_batches_out, int64_t* tel_out) {
+    return sorted_f_common_host(h, 2, order_out, batch_offsets_out, num_batches_out, tel_out);
 }
 
 int sched_sorted_f(sched_handle h, int32_t* order_out, int32_t* batch_offsets_out,

@@ -208,6 +208,32 @@ def test_sorted_f_local_swap_matches_oracle():
     assert total_swaps > 1000                                   # the improvement loop really ran
 
 
+def test_sorted_f_exact_dp_matches_oracle():
+    """Sorted-F with Algorithm 2 (exact DP) as Phase-1 solver: same batches, members and TEL as the
+    oracle's DP (which is itself checked against subset enumeration)."""
+    rng = np.random.default_rng(45)
+    cases = [W.tiny(), W.Instance("ex1", np.array([63] + [1] * 21, dtype=np.int32), np.array([1] + [2] * 21, dtype=np.int32), 64)]
+    for trial in range(25):
+        n = int(rng.integers(1, 60))
+        M = int(rng.integers(10, 400))
+        s, o = rand_instance(rng, n, M, M // 2, max(1, M // 3))
+        cases.append(W.Instance("rand", s, o, M))
+    big = W.mixed_backlog(100, 77, 16492, chat_s=(2.48, 1.58, 1, 4096), chat_o=(3.76, 1.17, 1, 2048), doc_s=(500, 4800), doc_o=(30, 560))
+    cases.append(big)                                           # the paper's recommended limit, n = 100
+    cases.append(W.Instance("ties", np.array([4, 4, 6, 8] * 12, dtype=np.int32), np.array([6, 6, 4, 2] * 12, dtype=np.int32), 50))
+    for inst in cases:
+        with kv.Scheduler(inst.s, inst.o, inst.M) as h:
+            order, offs, tel = h.sorted_f_dp()
+        r_order, r_offs = orc.sorted_f_exact(inst.s, inst.o, inst.M, orc.DP)
+        assert (offs == r_offs).all(), inst.name
+        assert (order == r_order).all(), inst.name
+        assert tel == orc.list_schedule_rounds(inst.s, inst.o, inst.M, r_order)[1]
+    with kv.Scheduler(np.ones(200, dtype=np.int32), np.ones(200, dtype=np.int32), 10) as h:
+        with pytest.raises(kv.SchedError) as e:
+            h.sorted_f_dp()
+        assert e.value.code == kv.E_UNSUPPORTED
+
+
 # ------------------------------------------------------------------------------------ POLICY
 def test_policy_sweep_small_batch():
     s, o, M = W.policy_sweep(num_instances=24, n_each=256)
