@@ -234,6 +234,30 @@ def test_sorted_f_exact_dp_matches_oracle():
         assert e.value.code == kv.E_UNSUPPORTED
 
 
+def test_tiny_backlog_all_solvers_and_brute_force():
+    """n = 16: prefix-F, Algorithm 4 and the exact DP orders, a full swap search from the DP order,
+    and all 8! orders of the first 8 requests against the oracle's brute force."""
+    import itertools
+    inst = W.tiny()
+    with kv.Scheduler(inst.s, inst.o, inst.M) as h:
+        o_dp, offs_dp, tel_dp = h.sorted_f_dp()
+        r_dp, r_offs = orc.sorted_f_exact(inst.s, inst.o, inst.M, orc.DP)
+        assert (o_dp == r_dp).all() and (offs_dp == r_offs).all()
+        final, tel, done, trace = h.local_search(kv.NBHD_SWAP, 100)       # starts from the DP order
+        r_final, r_tel, r_done, r_trace = orc.local_search(inst.s, inst.o, inst.M, orc.SWAP, 100, r_dp)
+        assert (final == r_final).all() and tel == r_tel and done == r_done and (trace == r_trace).all()
+        assert tel <= tel_dp
+    s8, o8 = inst.s[:8], inst.o[:8]
+    perms = np.array(list(itertools.permutations(range(8))), dtype=np.int32)
+    with kv.Scheduler(s8, o8, inst.M) as h:
+        tels, _, _ = h.eval_batch(kv.CAND_ORDER, perms)
+        dp8, _, tel8 = h.sorted_f_dp()
+    best, best_order = orc.bruteforce_best_order(s8, o8, inst.M)
+    assert tels.min() == best and (perms[int(np.argmin(tels))] == best_order).all()
+    opt, _ = orc.bruteforce_opt(s8, o8, inst.M, best + 1)
+    assert opt <= best <= tel8 < 48 * opt                              # Theorem 3's factor
+
+
 # ------------------------------------------------------------------------------------ POLICY
 def test_policy_sweep_small_batch():
     s, o, M = W.policy_sweep(num_instances=24, n_each=256)
