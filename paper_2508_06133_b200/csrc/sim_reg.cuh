@@ -29,9 +29,13 @@
 // relieves the pipe that limits this kernel.
 __constant__ int kv_const_one = 1;
 __device__ __forceinline__ int kv_add_fma_pipe(int a, int b) {
+#ifdef __CUDA_ARCH__
     int r;
     asm("mad.lo.s32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(kv_const_one), "r"(b));
     return r;
+#else
+    return a + b;
+#endif
 }
 
 // The passes over the window are specialised on a bucket (KLO, KHI] of the chunk count nch, chosen
@@ -60,6 +64,7 @@ struct RegSim {
     static constexpr int kWarps = NREG > 17 ? KV_REG33_WARPS : 32;
     int R[NREG];
     int t;
+    int tm, rl;              // t mod 32 and (lane - tm): window offset of this lane's cell of R[0]
     i64 tel;
 
     __device__ __forceinline__ void attach(int*, int) {}
@@ -68,7 +73,7 @@ struct RegSim {
     __device__ __forceinline__ void reset(int lane) {
 #pragma unroll
         for (int c = 0; c < NREG; ++c) R[c] = 32 * c + lane;
-        t = 0; tel = 0;
+        t = 0; tel = 0; tm = 0; rl = lane;
     }
 
     // snapshot layout: kCells ints, R[c] of lane l at [32 c + l]
@@ -76,6 +81,7 @@ struct RegSim {
 #pragma unroll
         for (int c = 0; c < NREG; ++c) R[c] = snap[32 * c + lane];
         t = h.t;
+        tm = t & 31; rl = lane - tm;
         tel = ((i64)h.tel_hi << 32) | (i64)(unsigned)h.tel_lo;
     }
 
@@ -129,7 +135,6 @@ struct RegSim {
     // registers rotate once per 32-round boundary crossed.  The rotation sits behind a real branch
     // (it is rare; as predicated moves it would cost NREG instructions on every call).
     __device__ __forceinline__ void advance(int delta, int lane) {
-        const int tm = t & 31, rl = lane - tm;
         const int step = min(delta, 32 - tm);
         if (rl >= 0 && rl < step) R[0] = t + rl + kCells;
         t += step;
@@ -141,6 +146,8 @@ struct RegSim {
             if (lane < delta) R[0] = t + lane + kCells;
             t += delta;
         }
+        tm = t & 31;
+        rl = lane - tm;
     }
 
     // Admit one request; returns its start.  All 32 lanes call this with identical (s, o).
@@ -162,14 +169,14 @@ struct RegSim {
             delta = pass_need<A, (B < NREG ? B : NREG)>(rl, ol, kadm);             \
         }
         {   // common case: the request fits at t
-            const int tm = t & 31, rl = lane - tm, ol = o - rl, nch = (tm + o + 31) >> 5;
+            const int ol = o - rl, nch = (tm + o + 31) >> 5;
             KV_RS_BUCKETS(nch, KV_RS_TRY)
         }
         for (int guard = 0;; ++guard) {
             delta = kv_warp_max(delta);                // >= 1: the worst cell alone asks for it
             kadm -= delta;
             advance(delta, lane);
-            const int tm = t & 31, rl = lane - tm, ol = o - rl, nch = (tm + o + 31) >> 5;
+            const int ol = o - rl, nch = (tm + o + 31) >> 5;
             KV_RS_BUCKETS(nch, KV_RS_TRY)
             if (guard > kCells) { if (lane == 0) atomicExch(status, KV_DEV_LOOP_CAP); return t; }
         }
