@@ -92,6 +92,14 @@ int sched_set_stream(sched_handle h, void* cuda_stream);
  * (SCHED_E_INTERNAL if any bounded loop gave up since the last call). */
 int sched_sync(sched_handle h);
 
+/* Prefill weight of the batch metric (Section 7, "Robustness to prefill weighting"):
+ * G(X) = sum (alpha * s_i + o_i) / |X|^2 with alpha = alpha_num / alpha_den; alpha = 0 (the default,
+ * 0/1) is the F-metric.  Applies to the following sched_sorted_f() and sched_sorted_f_local_swap()
+ * calls of this handle (in Algorithm 4 a swap then improves iff alpha*s_in + o_in < alpha*s_out +
+ * o_out); the exact DP and the POLICY candidates keep F.  Compared exactly on integer weights.
+ * SCHED_E_INVAL unless 0 <= alpha_num <= 2^20 and 1 <= alpha_den <= 2^20. */
+int sched_set_prefill_weight(sched_handle h, int32_t alpha_num, int32_t alpha_den);
+
 /* Base order used by SCHED_CAND_MOVE candidates and by sched_local_search(). host int32[n]. */
 int sched_set_base_order(sched_handle h, const int32_t* order);
 int sched_get_base_order(sched_handle h, int32_t* order_out);

@@ -219,3 +219,24 @@ def sorted_f_local_swap(s, o, M):
     if nb < 0:
         raise ValueError("a request exceeds M")
     return order, offs[:nb + 1].copy(), sw.value
+
+
+def _sorted_g(fn, s, o, M, a_num, a_den):
+    s, o = _i32(s), _i32(o)
+    n = len(s)
+    order = np.zeros(n, dtype=np.int32)
+    offs = np.zeros(n + 1, dtype=np.int32)
+    nb = fn(n, _p(s), _p(o), C.c_longlong(M), C.c_longlong(a_num), C.c_longlong(a_den), _p(order), _p(offs))
+    if nb < 0:
+        raise ValueError("bad weight or a request exceeds M")
+    return order, offs[:nb + 1].copy()
+
+
+def sorted_g_prefix(s, o, M, a_num, a_den):
+    """Sorted-G (metric sum(alpha*s+o)/k^2, alpha = a_num/a_den) with prefix batch selection."""
+    return _sorted_g(lib().orc_sorted_g_prefix, s, o, M, a_num, a_den)
+
+
+def sorted_g_local_swap(s, o, M, a_num, a_den):
+    """Sorted-G with Algorithm 4 as the batch solver."""
+    return _sorted_g(lib().orc_sorted_g_local_swap, s, o, M, a_num, a_den)

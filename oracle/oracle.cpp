@@ -567,4 +567,82 @@ int orc_sorted_f_local_swap(int n, const int* s, const int* o, i64 M, int* order
     return nb;
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// O11. Sorted-G (Section 7, "Robustness to prefill weighting"): the batch metric
+//      G(X) = sum (alpha * s_i + o_i) / |X|^2 with alpha = a_num / a_den >= 0; alpha = 0 is F.
+//      Compared exactly on the integer weights w_i = a_num * s_i + a_den * o_i (a common factor
+//      a_den does not change the order).  Everything else as in O6 (prefix selection) and O10
+//      (Algorithm 4, where a swap now improves iff w_in < w_out).
+// ---------------------------------------------------------------------------------------------
+int orc_sorted_g_prefix(int n, const int* s, const int* o, i64 M, i64 a_num, i64 a_den, int* order, int* batch_offsets) {
+    if (a_num < 0 || a_den <= 0) return -1;
+    std::vector<int> idx(n);
+    std::iota(idx.begin(), idx.end(), 0);
+    std::stable_sort(idx.begin(), idx.end(), [&](int a, int b) {
+        int ta = s[a] + o[a], tb = s[b] + o[b];
+        if (ta != tb) return ta < tb;
+        return o[a] < o[b];
+    });
+    int a = 0, nb = 0;
+    batch_offsets[0] = 0;
+    while (a < n) {
+        i64 mem = 0, sw = 0, bestSum = 0; int bestK = 0;
+        for (int k = 1; a + k <= n; ++k) {
+            int r = idx[a + k - 1];
+            mem += s[r] + o[r];
+            if (mem > M) break;
+            sw += a_num * s[r] + a_den * o[r];
+            if (bestK == 0 || orc_f_compare(sw, k, bestSum, bestK) < 0) { bestK = k; bestSum = sw; }
+        }
+        if (bestK == 0) return -1;
+        std::vector<int> X(idx.begin() + a, idx.begin() + a + bestK);
+        std::sort(X.begin(), X.end(), [&](int x, int y) { if (o[x] != o[y]) return o[x] < o[y]; return x < y; });
+        for (int k = 0; k < bestK; ++k) order[a + k] = X[k];
+        a += bestK;
+        batch_offsets[++nb] = a;
+    }
+    return nb;
+}
+
+int orc_sorted_g_local_swap(int n, const int* s, const int* o, i64 M, i64 a_num, i64 a_den, int* order, int* batch_offsets) {
+    if (a_num < 0 || a_den <= 0) return -1;
+    std::vector<int> rem(n);
+    std::iota(rem.begin(), rem.end(), 0);
+    int pos = 0, nb = 0;
+    batch_offsets[0] = 0;
+    while (!rem.empty()) {
+        const int m = (int)rem.size();
+        std::vector<int> I(rem);
+        std::stable_sort(I.begin(), I.end(), [&](int a, int b) { return s[a] + o[a] < s[b] + o[b]; });
+        std::vector<int> X, posX; std::vector<char> inX(m, 0);
+        i64 mem = 0;
+        for (int p = 0; p < m; ++p) { int r = I[p]; if (mem + s[r] + o[r] <= M) { X.push_back(r); posX.push_back(p); inX[p] = 1; mem += s[r] + o[r]; } }
+        if (X.empty()) return -1;
+        bool improved = true;
+        while (improved) {
+            improved = false;
+            for (size_t k = 0; k < X.size() && !improved; ++k) {
+                int rout = X[k];
+                for (int p = 0; p < m; ++p) {
+                    if (inX[p]) continue;
+                    int rin = I[p];
+                    i64 dm = (i64)(s[rin] + o[rin]) - (s[rout] + o[rout]);
+                    if (mem + dm > M) continue;
+                    i64 dw = (a_num * s[rin] + a_den * o[rin]) - (a_num * s[rout] + a_den * o[rout]);
+                    if (dw < 0) { inX[posX[k]] = 0; inX[p] = 1; posX[k] = p; X[k] = rin; mem += dm; improved = true; break; }
+                }
+            }
+        }
+        std::sort(X.begin(), X.end(), [&](int a, int b) { if (o[a] != o[b]) return o[a] < o[b]; return a < b; });
+        std::vector<char> gone(n, 0);
+        for (int x : X) { order[pos++] = x; gone[x] = 1; }
+        batch_offsets[++nb] = pos;
+        std::vector<int> rest;
+        for (int r : rem) if (!gone[r]) rest.push_back(r);
+        rem.swap(rest);
+    }
+    return nb;
+}
+
 }  // extern "C"

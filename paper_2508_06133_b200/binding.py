@@ -20,7 +20,7 @@ POLICY_FCFS, POLICY_SOF, POLICY_TOTAL_SIZE, POLICY_SORTED_F = 0, 1, 2, 3
 NBHD_SWAP, NBHD_SWAP_INSERT, NBHD_SAMPLED = 0, 1, 2
 
 EXPORTS = [
-    "sched_init", "sched_init_batch", "sched_set_stream", "sched_sync", "sched_set_base_order",
+    "sched_init", "sched_init_batch", "sched_set_stream", "sched_sync", "sched_set_prefill_weight", "sched_set_base_order",
     "sched_get_base_order", "sched_eval_batch", "sched_eval_batch_dev", "sched_sweep_dev",
     "sched_sorted_f", "sched_sorted_f_dev", "sched_sorted_f_local_swap", "sched_sorted_f_local_swap_dev", "sched_sorted_f_dp", "sched_local_search", "sched_last_eval_kernel_ms", "sched_argmin_static_dev", "sched_stats", "sched_destroy",
     "sched_strerror", "sched_last_cuda_error",
@@ -57,6 +57,7 @@ def load():
     lib.sched_set_stream.argtypes = [vp, vp]
     lib.sched_sync.argtypes = [vp]
     lib.sched_set_base_order.argtypes = [vp, vp]
+    lib.sched_set_prefill_weight.argtypes = [vp, i32, i32]
     lib.sched_get_base_order.argtypes = [vp, vp]
     lib.sched_eval_batch.argtypes = [vp, C.c_int, i64, vp, vp, vp, vp]
     lib.sched_eval_batch_dev.argtypes = [vp, C.c_int, i64, vp, vp, vp, vp]
@@ -160,6 +161,10 @@ class Scheduler:
         ms = C.c_float(0)
         _check(load().sched_last_eval_kernel_ms(self._h, C.byref(ms)), "sched_last_eval_kernel_ms")
         return ms.value
+
+    def set_prefill_weight(self, alpha_num, alpha_den=1):
+        """Batch metric G = sum(alpha*s + o)/k^2 with alpha = alpha_num/alpha_den (0: the F-metric)."""
+        _check(load().sched_set_prefill_weight(self._h, alpha_num, alpha_den), "sched_set_prefill_weight")
 
     def set_base_order(self, order):
         order = np.ascontiguousarray(order, dtype=np.int32)

@@ -176,6 +176,7 @@ int create_common(sched_ctx** out, int B, int n, const int32_t* s, const int32_t
         h->sm_count = prop.multiProcessorCount;
         h->smem_optin = (int)prop.sharedMemPerBlockOptin;
         h->B = B; h->n = n; h->M = M; h->omax = omax; h->sum_o_max = sum_max;
+        h->g_num = 0; h->g_den = 1;
         h->nreg = sim_pick_nreg(omax);
         if (const char* kind = getenv("KVSCHED_SIM"))               // testing knob: "smem" forces the shared-memory simulator
             if (strcmp(kind, "smem") == 0) h->nreg = 0;
@@ -395,6 +396,13 @@ int sched_sync(sched_handle h) {
     return read_status(h);
 }
 
+int sched_set_prefill_weight(sched_handle h, int32_t alpha_num, int32_t alpha_den) {
+    if (!h) return SCHED_E_INVAL;
+    if (alpha_num < 0 || alpha_den < 1 || alpha_num > (1 << 20) || alpha_den > (1 << 20)) return SCHED_E_INVAL;
+    h->g_num = alpha_num; h->g_den = alpha_den;
+    return SCHED_OK;
+}
+
 int sched_set_base_order(sched_handle h, const int32_t* order) {
     KV_ENTER(h);
     if (h->batch_handle || !order) return SCHED_E_INVAL;
@@ -591,7 +599,8 @@ static int sorted_f_common_dev(sched_handle h, int solver, int32_t* order_out, i
                                                           key_byte_mask(bits_of((u64)h->omax), bits_of((u64)h->M)));
         KV_TRY(check_launch(h));
         // S2: prefix sums + F-metric batch boundaries
-        k2_prefix_f<<<1, 1024, 0, st>>>(h->d_s, h->d_o, h->d_vals_a, n, h->M, h->d_prefP, h->d_prefO, h->d_batch_off, h->d_num_batches);
+        k2_prefix_f<<<1, 1024, 0, st>>>(h->d_s, h->d_o, h->d_vals_a, n, h->M, h->d_prefP, h->d_prefO, h->d_batch_off, h->d_num_batches,
+                                        (i64)h->g_num, (i64)h->g_den);
         KV_TRY(check_launch(h));
     } else if (solver == 2) {
         KV_TRY(phase1_dp(h));
@@ -604,7 +613,8 @@ static int sorted_f_common_dev(sched_handle h, int solver, int32_t* order_out, i
                                                           key_byte_mask(0, bits_of((u64)h->M)));
         KV_TRY(check_launch(h));
         int* ls = h->d_ls;
-        k2_local_swap<<<1, K2L_THREADS, 0, st>>>(h->d_s, h->d_o, h->d_vals_a, n, h->M, ls, ls + n, ls + 2 * (size_t)n,
+        if ((i64)h->g_num * h->M + (i64)h->g_den * h->omax >= (1ll << 31)) return SCHED_E_UNSUPPORTED;   // 32-bit weights
+        k2_local_swap<<<1, K2L_THREADS, 0, st>>>(h->d_s, h->d_o, h->d_vals_a, n, h->M, h->g_num, h->g_den, ls, ls + n, ls + 2 * (size_t)n,
                                                  ls + 3 * (size_t)n, ls + 4 * (size_t)n, ls + 5 * (size_t)n, ls + 6 * (size_t)n,
                                                  h->d_vals_b, h->d_batch_off, h->d_num_batches, h->d_status);
         KV_TRY(check_launch(h));

@@ -46,6 +46,7 @@ struct sched_ctx {
     void* h_pinned;          // 64 bytes of pinned host memory for small read-backs
     void* d_sort;            // grow-only scratch for sorting explicit start times
     size_t sort_cap;
+    int g_num, g_den;        // prefill weight alpha = g_num / g_den of the batch metric (0/1: the F-metric)
     int* d_ls;               // scratch of the Local Swap Search kernel: 7 arrays of n ints (lazy)
     void* d_k4;              // grow-only scratch of the launch ordering: bins[n+1], first_pos[count], order[count]
     size_t k4_cap;

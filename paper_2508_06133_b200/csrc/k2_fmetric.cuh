@@ -30,16 +30,19 @@ __device__ __forceinline__ bool k2_f_better(u64 sumA, u64 kA, u64 sumB, u64 kB) 
 
 // Inclusive-to-exclusive prefix sums of T = s+o and o over `ids` (list order):
 // P[0] = O[0] = 0, P[q+1] = P[q] + T(ids[q]).  Block-wide, chunked; `carry` is 2 shared words.
+// With a prefill weight alpha = a_num / a_den (Section 7's G-metric, alpha = 0 is F) the second sum
+// runs over a_num * s + a_den * o instead of o.
 __device__ void k2_prefix_sums(const int* __restrict__ s, const int* __restrict__ o,
                                const int* __restrict__ ids, int n, i64* P, i64* O,
-                               i64* sh_warp /* [2 * 32] */, i64* carry /* [2] */) {
+                               i64* sh_warp /* [2 * 32] */, i64* carry /* [2] */,
+                               i64 a_num = 0, i64 a_den = 1) {
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5, nw = blockDim.x >> 5;
     if (tid == 0) { carry[0] = 0; carry[1] = 0; P[0] = 0; O[0] = 0; }
     __syncthreads();
     for (int base = 0; base < n; base += blockDim.x) {
         const int q = base + tid;
         i64 vt = 0, vo = 0;
-        if (q < n) { int id = ids[q]; vo = o[id]; vt = (i64)s[id] + vo; }
+        if (q < n) { int id = ids[q]; vt = (i64)s[id] + o[id]; vo = a_num * s[id] + a_den * o[id]; }
         i64 it = vt, io = vo;
         for (int d = 1; d < 32; d <<= 1) {
             i64 yt = __shfl_up_sync(KV_FULL, it, d), yo = __shfl_up_sync(KV_FULL, io, d);
@@ -110,11 +113,11 @@ __device__ int k2_select_batches(const i64* P, const i64* O, int n, i64 M, int* 
 __global__ void __launch_bounds__(1024)
 k2_prefix_f(const int* __restrict__ s, const int* __restrict__ o, const int* __restrict__ sorted_ids,
             int n, i64 M, i64* __restrict__ P, i64* __restrict__ O,
-            int* __restrict__ batch_off, int* __restrict__ num_batches) {
+            int* __restrict__ batch_off, int* __restrict__ num_batches, i64 a_num, i64 a_den) {
     __shared__ i64 sh_warp[64];
     __shared__ i64 carry[2];
     __shared__ u64 sh_best[66];
-    k2_prefix_sums(s, o, sorted_ids, n, P, O, sh_warp, carry);
+    k2_prefix_sums(s, o, sorted_ids, n, P, O, sh_warp, carry, a_num, a_den);
     __syncthreads();
     int nb = k2_select_batches(P, O, n, M, batch_off, sh_best);
     if (threadIdx.x == 0) *num_batches = nb;

@@ -8,7 +8,8 @@
 //   improvement -- walk r_out over X (insertion order, a swapped-in request keeps the place of the
 //                 one it replaces) and r_in over the requests outside X (sorted order); the first
 //                 pair with  mem + (s+o)_in - (s+o)_out <= M  and  F(X') < F(X)  is swapped and the
-//                 walk starts over; |X| never changes, so F drops iff o_in < o_out.
+//                 walk starts over; |X| never changes, so F drops iff o_in < o_out (with Section 7's
+//                 prefill weight alpha = a_num / a_den: iff a_num s_in + a_den o_in is smaller).
 // The pair walk is not executed cell by cell.  For one r_out the admissible r_in are the outside
 // requests among the first ub positions (sizes ascend: (s+o)_in <= cap is a prefix), and the first
 // of them with o_in < o_out is the first position where the running minimum of o over outside
@@ -51,7 +52,7 @@ __device__ __forceinline__ int k2l_first_below(const int* a, int len, int thr) {
 // order_out receives every batch in X's walking order (the caller sorts each batch by (o, index)).
 __global__ void __launch_bounds__(K2L_THREADS)
 k2_local_swap(const int* __restrict__ s, const int* __restrict__ o, const int* __restrict__ sorted_ids,
-              int n, i64 M, int* removed, int* rem, int* remT, int* remO, int* inX, int* pm, int* xpos,
+              int n, i64 M, int a_num, int a_den, int* removed, int* rem, int* remT, int* remO, int* inX, int* pm, int* xpos,
               int* __restrict__ order_out, int* __restrict__ batch_off, int* __restrict__ num_batches,
               int* status) {
     __shared__ i64 sh64[33];
@@ -78,7 +79,7 @@ k2_local_swap(const int* __restrict__ s, const int* __restrict__ o, const int* _
             if (f) {
                 const int p = m + before + incl - 1;
                 const int id = sorted_ids[i];
-                rem[p] = i; remT[p] = s[id] + o[id]; remO[p] = o[id];
+                rem[p] = i; remT[p] = s[id] + o[id]; remO[p] = a_num * s[id] + a_den * o[id];   // weight: o when alpha = 0
             }
             m += total;
             __syncthreads();

@@ -258,6 +258,31 @@ def test_tiny_backlog_all_solvers_and_brute_force():
     assert opt <= best <= tel8 < 48 * opt                              # Theorem 3's factor
 
 
+def test_sorted_g_prefill_weight_matches_oracle():
+    rng = np.random.default_rng(46)
+    cases = [W.mixed_1k(), W.paper_scale()]
+    for trial in range(20):
+        n = int(rng.integers(1, 300))
+        M = int(rng.integers(10, 1500))
+        s, o = rand_instance(rng, n, M, M // 2, max(1, M // 3))
+        cases.append(W.Instance("rand", s, o, M))
+    for inst in cases:
+        with kv.Scheduler(inst.s, inst.o, inst.M) as h:
+            for a_num, a_den in ((1, 1), (13, 1000), (5, 1), (0, 3)):
+                h.set_prefill_weight(a_num, a_den)
+                order, offs, tel = h.sorted_f()
+                r_order, r_offs = orc.sorted_g_prefix(inst.s, inst.o, inst.M, a_num, a_den)
+                assert (offs == r_offs).all() and (order == r_order).all(), (inst.name, a_num, a_den)
+                assert tel == orc.list_schedule_rounds(inst.s, inst.o, inst.M, r_order)[1]
+                order, offs, tel = h.sorted_f_local_swap()
+                r_order, r_offs = orc.sorted_g_local_swap(inst.s, inst.o, inst.M, a_num, a_den)
+                assert (offs == r_offs).all() and (order == r_order).all(), (inst.name, a_num, a_den)
+            with pytest.raises(kv.SchedError):
+                h.set_prefill_weight(-1, 1)
+            with pytest.raises(kv.SchedError):
+                h.set_prefill_weight(1, 0)
+
+
 # ------------------------------------------------------------------------------------ POLICY
 def test_policy_sweep_small_batch():
     s, o, M = W.policy_sweep(num_instances=24, n_each=256)

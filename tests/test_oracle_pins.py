@@ -462,3 +462,47 @@ def test_local_swap_example1_and_properties(golden):
         for a, b in zip(offs[:-1], offs[1:]):
             assert (np.diff(o[order[a:b]]) >= 0).all() and int(T[order[a:b]].sum()) <= M
         assert order[:offs[1]].tolist() == sorted(X.tolist(), key=lambda i: (o[i], i))
+
+
+# ----------------------------------------------------------------------------- Sorted-G (prefill-weighted metric)
+def test_sorted_g_reduces_to_f_and_differs_by_hand():
+    from fractions import Fraction
+    rng = np.random.default_rng(606)
+    for trial in range(60):
+        n = int(rng.integers(1, 60))
+        M = int(rng.integers(10, 300))
+        s, o = random_instance(rng, n, M, M // 2, M // 3 + 1)
+        # alpha = 0 recovers the F-metric (Section 7), whatever the denominator
+        for den in (1, 7):
+            og, fg = orc.sorted_g_prefix(s, o, M, 0, den)
+            of, ff = orc.sorted_f_prefix(s, o, M)
+            assert (og == of).all() and (fg == ff).all()
+            og, fg = orc.sorted_g_local_swap(s, o, M, 0, den)
+            ol, fl, _ = orc.sorted_f_local_swap(s, o, M)
+            assert (og == ol).all() and (fg == fl).all()
+        # first batch against the definition with exact fractions: G(X) = sum(alpha*s+o)/|X|^2
+        a_num, a_den = int(rng.integers(0, 6)), int(rng.integers(1, 5))
+        alpha = Fraction(a_num, a_den)
+        order, offs = orc.sorted_g_prefix(s, o, M, a_num, a_den)
+        by_size = sorted(range(n), key=lambda i: (int(s[i]) + int(o[i]), int(o[i]), i))
+        best, best_k, mem, tot = None, 0, 0, Fraction(0)
+        for k, i in enumerate(by_size, 1):
+            mem += int(s[i]) + int(o[i])
+            if mem > M:
+                break
+            tot += alpha * int(s[i]) + int(o[i])
+            g = tot / (k * k)
+            if best is None or g < best or (g == best and k > best_k):
+                best, best_k = g, k
+        assert offs[1] == best_k and sorted(order[:best_k].tolist()) == sorted(by_size[:best_k])
+    # by hand: B(1,4) B(1,4) A(30,1), M = 41.  F: 4/1, 8/4, 9/9 -> all three.  alpha = 1: 5/1, 10/4,
+    # 41/9 -> only the two small prompts.
+    s, o = np.array([30, 1, 1], dtype=np.int32), np.array([1, 4, 4], dtype=np.int32)
+    assert orc.sorted_g_prefix(s, o, 41, 0, 1)[1].tolist() == [0, 3]
+    assert orc.sorted_g_prefix(s, o, 41, 1, 1)[1].tolist() == [0, 2, 3]
+    # Algorithm 4 under G: swapping in the long prompt A(30,1) for B lowers sum(o) but not sum(s+o)
+    s, o = np.array([1, 1, 3], dtype=np.int32), np.array([4, 4, 1], dtype=np.int32)      # sizes 5, 5, 4; M = 9
+    assert sorted(orc.sorted_f_local_swap(s, o, 9)[0][:2].tolist()) == [0, 2]            # first fit {2,0}; nothing better
+    s, o = np.array([1, 1, 4], dtype=np.int32), np.array([4, 4, 1], dtype=np.int32)      # sizes 5, 5, 5; M = 10
+    assert sorted(orc.sorted_f_local_swap(s, o, 10)[0][:2].tolist()) == [1, 2]           # F: o 1 < 4 -> swap request 0 out
+    assert sorted(orc.sorted_g_local_swap(s, o, 10, 1, 1)[0][:2].tolist()) == [0, 1]     # G, alpha=1: weights 5,5,5 -> no swap
