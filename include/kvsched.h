@@ -118,7 +118,10 @@ int sched_get_base_order(sched_handle h, int32_t* order_out);
 int sched_eval_batch(sched_handle h, int kind, int64_t count, const void* candidates,
                      int64_t* tel_out, uint8_t* feasible_out, int32_t* starts_out);
 
-/* Same, device pointers, asynchronous on the handle's stream, candidates not validated. */
+/* Same, device pointers, asynchronous on the handle's stream.  Candidates are not validated on the
+ * host; a MOVE code outside the neighbourhood or an ORDER entry outside 0..n-1 yields
+ * tel_out = INT64_MAX for that candidate (duplicate ids in an ORDER are not detected), a negative
+ * start time yields feasible_out = 0. */
 int sched_eval_batch_dev(sched_handle h, int kind, int64_t count, const void* candidates,
                          int64_t* tel_out, uint8_t* feasible_out, int32_t* starts_out);
 

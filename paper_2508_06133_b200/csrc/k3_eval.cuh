@@ -168,6 +168,10 @@ k3_eval_moves(const MoveEvalParams p) {
     SIM sim;
     sim.attach((int*)(smem_raw + ring_off) + (size_t)warp * L, L);
     const Move mv = k4_move_of(p.src, n, c);
+    if ((unsigned)mv.i >= (unsigned)n || (unsigned)mv.j >= (unsigned)n) {      // code outside the neighbourhood
+        if (lane == 0) p.tel_out[c] = INT64_MAX;
+        return;
+    }
     const int first_pos = min(mv.i, mv.j);
     const int idx = first_pos / p.stride;
     const int q_start = idx * p.stride;
@@ -232,11 +236,16 @@ k3_eval_orders(const OrderEvalParams p) {
     const int* ord = p.orders + (size_t)c * n;
     int* starts = kStarts ? p.starts_out + (size_t)c * n : nullptr;
     sim.reset(lane);
+    int bad = 0;
     for (int q0 = 0; q0 < n; q0 += 32) {
         const int qq = q0 + lane;
         int2 so = make_int2(1, 1);
         int id = 0;
-        if (qq < n) { id = ord[qq]; so = tbl[id]; }
+        if (qq < n) { id = ord[qq]; if ((unsigned)id >= (unsigned)n) { id = 0; bad = 1; } so = tbl[id]; }
+        if (__any_sync(KV_FULL, bad)) {                                       // an id outside 0..n-1
+            if (lane == 0) p.tel_out[c] = INT64_MAX;
+            return;
+        }
         const int cnt = min(32, n - q0);
         for (int k = 0; k < cnt; ++k) {
             const int s = __shfl_sync(KV_FULL, so.x, k), o = __shfl_sync(KV_FULL, so.y, k);
@@ -380,6 +389,7 @@ k3_check_starts(const StartsEvalParams p) {
                 if (!ok) continue;
                 // advance the ring to round pk: cells of rounds t .. pk-1 are finished
                 const int adv = pk - t;
+                if (adv < 0) { ok = false; continue; }                       // starts not ascending: unsorted or negative input
                 if (adv >= L) { for (int r = lane; r < L; r += 32) ring[r] = 0; }
                 else for (int r = lane; r < adv; r += 32) ring[kv_wrap(tr + r, L)] = 0;
                 __syncwarp();

@@ -33,7 +33,8 @@ __global__ void k4_first_pos_histogram(MoveSource src, int n, i64 count, int* __
     const i64 c = (i64)blockIdx.x * blockDim.x + threadIdx.x;
     if (c >= count) return;
     const Move m = k4_move_of(src, n, c);
-    const int fp = min(m.i, m.j);
+    int fp = min(m.i, m.j);
+    if (fp < 0 || fp >= n) fp = n - 1;               // invalid code: the evaluator rejects it, any bucket will do
     first_pos[c] = fp;
     atomicAdd(&bins[fp], 1);
 }

@@ -391,6 +391,33 @@ def test_local_search_first_sweeps_mixed_1k():
     assert oracle_moves(inst.s, inst.o, inst.M, base, codes).min() >= trace[0][1]
 
 
+def test_device_pointer_candidates_are_bounds_checked_on_the_device():
+    import torch
+    dev = torch.device("cuda", torch.cuda.current_device())
+    s, o = np.array([2, 3, 4, 5], dtype=np.int32), np.array([1, 2, 3, 1], dtype=np.int32)
+    big = np.iinfo(np.int64).max
+    with kv.Scheduler(s, o, 20) as h:
+        codes = torch.tensor([0, 17, 18, 10 ** 12, -5], dtype=torch.int64, device=dev)     # 6 swaps + 12 inserts: 0..17 valid
+        tel = torch.zeros(5, dtype=torch.int64, device=dev)
+        h.eval_batch_dev(kv.CAND_MOVE, 5, codes, tel)
+        h.sync()
+        got = tel.cpu().numpy()
+        assert got[0] == oracle_moves(s, o, 20, np.arange(4), [0])[0] and got[1] == oracle_moves(s, o, 20, np.arange(4), [17])[0]
+        assert (got[2:] == big).all()
+        orders = torch.tensor([[3, 2, 1, 0], [0, 1, 2, 4], [0, -1, 2, 3]], dtype=torch.int32, device=dev)
+        tel = torch.zeros(3, dtype=torch.int64, device=dev)
+        h.eval_batch_dev(kv.CAND_ORDER, 3, orders, tel)
+        h.sync()
+        got = tel.cpu().numpy()
+        assert got[0] == orc.list_schedule_alg1(s, o, 20, [3, 2, 1, 0])[1] and (got[1:] == big).all()
+        starts = torch.tensor([[0, 0, 0, 0], [0, -3, 0, 0]], dtype=torch.int32, device=dev)
+        tel = torch.zeros(2, dtype=torch.int64, device=dev)
+        feas = torch.zeros(2, dtype=torch.uint8, device=dev)
+        h.eval_batch_dev(kv.CAND_START_TIMES, 2, starts, tel, feas)
+        h.sync()
+        assert feas.cpu().numpy().tolist() == [int(orc.check_schedule(s, o, 20, [0, 0, 0, 0])["feasible"]), 0]
+
+
 # ------------------------------------------------------------------------------------ errors on a live handle
 def test_error_paths_on_a_handle():
     s, o = np.array([2, 3, 4], dtype=np.int32), np.array([1, 2, 3], dtype=np.int32)
