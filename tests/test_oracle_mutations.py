@@ -1,0 +1,70 @@
+"""Do the pins bite?  Each case plants one plausible mistake in a copy of the CPU oracle (never in
+the GPU code), loads the mutated library in place of the real one and checks that a named pin test
+fails.  A pin that still passed would mean that part of the oracle is effectively unpinned."""
+import ctypes as C
+import os
+import subprocess
+
+import pytest
+
+import oracle as orc
+from tests import test_oracle_pins as pins
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+SRC = os.path.join(os.path.dirname(HERE), "oracle", "oracle.cpp")
+
+MUTATIONS = [
+    # (what, text in oracle.cpp, replacement, pin that must fail, needs the golden fixture)
+    ("start-time convention of Algorithm 1", "p[i] = t - 1;", "p[i] = t;", "test_example1_tel", True),
+    ("capacity off by one in the round-form executor", "if (U[k + j] + s[i] + j > M) { fits = false; break; }",
+     "if (U[k + j] + s[i] + j >= M) { fits = false; break; }", "test_example1_tel", True),
+    ("ramp term dropped in the checker", "U[p[i] + j] += (i64)s[i] + j;\n    i64 pk", "U[p[i] + j] += (i64)s[i];\n    i64 pk",
+     "test_example1_checker_by_hand", True),
+    ("completion time without the decode length", "for (int i = 0; i < n; ++i) total += p[i] + o[i];\n    if (tel) *tel = total;\n    if (peak)",
+     "for (int i = 0; i < n; ++i) total += p[i];\n    if (tel) *tel = total;\n    if (peak)", "test_example1_checker_by_hand", True),
+    ("F ties to the smaller batch", "if (kA != kB) return kA > kB ? -1 : 1;", "if (kA != kB) return kA < kB ? -1 : 1;",
+     "test_example1_f_metric", True),
+    ("F compared with k instead of k^2", "u128 l = (u128)sumA * (u128)kB * (u128)kB, r = (u128)sumB * (u128)kA * (u128)kA;",
+     "u128 l = (u128)sumA * (u128)kB, r = (u128)sumB * (u128)kA;", "test_phase1_dp_matches_enumeration_and_lemma1", False),
+    ("prefix-F memory test off by one", "mem += s[r] + o[r];\n            if (mem > M) break;\n            so += o[r];",
+     "mem += s[r] + o[r];\n            if (mem >= M) break;\n            so += o[r];", "test_prefix_f_by_hand", False),
+    ("insert code maps to the wrong target", "*type = 1; *i_out = i; *j_out = r < i ? r : r + 1;",
+     "*type = 1; *i_out = i; *j_out = r <= i ? r : r + 1;", "test_move_codes_enumerate_the_neighbourhood", False),
+    ("Algorithm 4 memory test off by one", "if (mem + dm > M) continue;\n                i64 d_o",
+     "if (mem + dm >= M) continue;\n                i64 d_o", "test_local_swap_worked_by_hand", False),
+    ("G-metric without the prefill term", "sw += a_num * s[r] + a_den * o[r];", "sw += a_den * o[r];",
+     "test_sorted_g_reduces_to_f_and_differs_by_hand", False),
+    ("shortest-output-first sorts by size", "std::stable_sort(order, order + n, [&](int a, int b) { return o[a] < o[b]; });",
+     "std::stable_sort(order, order + n, [&](int a, int b) { return s[a] + o[a] < s[b] + o[b]; });", "test_policies", False),
+]
+
+
+@pytest.fixture(scope="module")
+def source():
+    return open(SRC).read()
+
+
+@pytest.mark.parametrize("what,old,new,pin,needs_golden", MUTATIONS, ids=[m[0] for m in MUTATIONS])
+def test_pin_catches_planted_mistake(tmp_path, source, golden, what, old, new, pin, needs_golden):
+    assert source.count(old) == 1, "mutation site must be unique: " + what
+    mutated = tmp_path / "oracle_mut.cpp"
+    mutated.write_text(source.replace(old, new))
+    so = tmp_path / "liboracle_mut.so"
+    subprocess.check_call(["g++", "-O1", "-std=c++17", "-shared", "-fPIC", "-o", str(so), str(mutated)])
+    lib = C.CDLL(str(so))
+    lib.orc_bruteforce_opt.restype = C.c_longlong
+    lib.orc_bruteforce_best_order.restype = C.c_longlong
+    real = orc.lib()
+    fn = getattr(pins, pin)
+    orc._lib = lib
+    try:
+        with pytest.raises((AssertionError, ValueError)):
+            if pin == "test_example1_tel":
+                for ex in (orc.list_schedule_alg1, orc.list_schedule_rounds):
+                    fn(golden, ex)
+            elif needs_golden:
+                fn(golden)
+            else:
+                fn()
+    finally:
+        orc._lib = real
