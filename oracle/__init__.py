@@ -240,3 +240,43 @@ def sorted_g_prefix(s, o, M, a_num, a_den):
 def sorted_g_local_swap(s, o, M, a_num, a_den):
     """Sorted-G with Algorithm 4 as the batch solver."""
     return _sorted_g(lib().orc_sorted_g_local_swap, s, o, M, a_num, a_den)
+
+
+def quantile_greedy_batch(ids, s, o, M, sample):
+    """Algorithm 5 on the request set ``ids`` with the given sample.
+    Returns (X in admission order, Q_p, Q_o)."""
+    s, o, ids, sample = _i32(s), _i32(o), _i32(ids), _i32(sample)
+    chosen = np.zeros(len(ids), dtype=np.int32)
+    qp, qo = C.c_longlong(0), C.c_longlong(0)
+    c = lib().orc_quantile_greedy_batch(len(ids), _p(ids), _p(s), _p(o), C.c_longlong(M), len(sample), _p(sample),
+                                        _p(chosen), C.byref(qp), C.byref(qo))
+    if c <= 0:
+        raise ValueError("empty input, empty sample or a request that exceeds M")
+    return chosen[:c].copy(), qp.value, qo.value
+
+
+def quantile_sample(ids, o, seed, batch):
+    """The reproducible 'random subset' of Algorithm 5 for batch number ``batch``."""
+    o, ids = _i32(o), _i32(ids)
+    out = np.zeros(max(1, len(ids)), dtype=np.int32)
+    c = lib().orc_quantile_sample(len(ids), _p(ids), _p(o), C.c_uint64(seed), int(batch), _p(out))
+    return out[:c].copy()
+
+
+def sorted_f_quantile(s, o, M, seed):
+    """Sorted-F with Algorithm 5 as Phase-1 solver.  Returns (order, batch offsets)."""
+    s, o = _i32(s), _i32(o)
+    n = len(s)
+    order = np.zeros(n, dtype=np.int32)
+    offs = np.zeros(n + 1, dtype=np.int32)
+    nb = lib().orc_sorted_f_quantile(n, _p(s), _p(o), C.c_longlong(M), C.c_uint64(seed), _p(order), _p(offs))
+    if nb < 0:
+        raise ValueError("a request exceeds M")
+    return order, offs[: nb + 1].copy()
+
+
+def mix64(z):
+    """One splitmix64 step from state ``z`` (the generator behind every sampled quantity)."""
+    f = lib().orc_mix64
+    f.restype = C.c_uint64
+    return int(f(C.c_uint64(z & 0xFFFFFFFFFFFFFFFF)))

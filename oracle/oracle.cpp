@@ -2,7 +2,9 @@
 //
 // A plain, slow, single-threaded restatement of what the paper defines: the memory model and
 // total end-to-end latency (Section 2.1-2.2, integer program of Section 6.1), the F-metric and
-// Sorted-F (Section 3, Algorithm 1), the exact dynamic programme (Section 5.1, Algorithm 2), and
+// Sorted-F (Section 3, Algorithm 1), the exact dynamic programme (Section 5.1, Algorithm 2),
+// Local Swap Search and Quantile Greedy Selection (Sections 5.2-5.3, Algorithms 4 and 5),
+// Sorted-G (Section 7), and
 // an order-level local search that scores every neighbour with Algorithm 1's Phase 2.  It exists
 // so that the GPU library can be checked against it; it shares no code with that library, is never
 // called by it, and nothing here is tuned for speed.  All arithmetic is integer.
@@ -15,7 +17,10 @@
 //
 // Parity status: every function below is pinned by tests that do not go through this file's own
 // formulas (paper's worked example, closed forms, brute force), except where marked
-// "parity unpinned".
+// "parity unpinned".  O12 (Algorithm 5): the routine is pinned for a GIVEN sample (hand-worked
+// cases, a library quantile, maximality), and the sampling hash to the generator's published
+// values; but which subset "random subset" means and how the 0.3-quantile of a finite sample is
+// read are choices no printed value fixes -- for those two choices: parity unpinned.
 #include <algorithm>
 #include <cstdint>
 #include <cstring>
@@ -375,6 +380,8 @@ static uint64_t mix64(uint64_t z) {
     return z ^ (z >> 31);
 }
 
+uint64_t orc_mix64(uint64_t z) { return mix64(z); }
+
 void orc_sample_move(int n, uint64_t seed, int it, i64 m, int* type, int* i_out, int* j_out) {
     uint64_t h1 = mix64(seed ^ mix64(((uint64_t)(uint32_t)it << 32) + (uint64_t)m));
     uint64_t h2 = mix64(h1);
@@ -634,6 +641,94 @@ int orc_sorted_g_local_swap(int n, const int* s, const int* o, i64 M, i64 a_num,
                 }
             }
         }
+        std::sort(X.begin(), X.end(), [&](int a, int b) { if (o[a] != o[b]) return o[a] < o[b]; return a < b; });
+        std::vector<char> gone(n, 0);
+        for (int x : X) { order[pos++] = x; gone[x] = 1; }
+        batch_offsets[++nb] = pos;
+        std::vector<int> rest;
+        for (int r : rem) if (!gone[r]) rest.push_back(r);
+        rem.swap(rest);
+    }
+    return nb;
+}
+
+
+// ---------------------------------------------------------------------------------------------
+// O12. Algorithm 5 (Quantile Greedy Selection): one batch out of the request set `ids`.
+//      I = ids sorted by ascending o (ties: lower index).  Q_p and Q_o are the 0.3-quantiles of
+//      s+o and of o over `sample`.  Pass 1 walks I and admits r when s_r+o_r <= Q_p, o_r <= Q_o
+//      and it still fits (mem + s_r + o_r <= M).  Pass 2 walks the requests left over, sorted by
+//      ascending o/(s+o), and admits every one that still fits.
+//      Left open by the listing and fixed here: the q-quantile of m values is the element at
+//      0-based position floor(q (m-1)) of the ascending values (no interpolation; 0.3 = 3/10 in
+//      integers); both sorts are stable, so equal o/(s+o) keep their order in I; the ratio is
+//      compared exactly (o_a (s_b+o_b) < o_b (s_a+o_a)).
+// Writes X in admission order, returns |X|; qp_out/qo_out (nullable) receive the thresholds.
+// ---------------------------------------------------------------------------------------------
+int orc_quantile_greedy_batch(int m, const int* ids, const int* s, const int* o, i64 M,
+                              int sample_size, const int* sample, int* chosen, i64* qp_out, i64* qo_out) {
+    if (m <= 0 || sample_size <= 0) return -1;
+    std::vector<int> I(ids, ids + m);
+    std::stable_sort(I.begin(), I.end(), [&](int a, int b) { if (o[a] != o[b]) return o[a] < o[b]; return a < b; });
+    std::vector<i64> vp, vo;
+    for (int k = 0; k < sample_size; ++k) { vp.push_back((i64)s[sample[k]] + o[sample[k]]); vo.push_back(o[sample[k]]); }
+    std::sort(vp.begin(), vp.end());
+    std::sort(vo.begin(), vo.end());
+    const int q = (int)((3ll * (sample_size - 1)) / 10);
+    const i64 Qp = vp[q], Qo = vo[q];
+    if (qp_out) *qp_out = Qp;
+    if (qo_out) *qo_out = Qo;
+    std::vector<int> X, remaining;
+    i64 mem = 0;
+    for (int r : I) {
+        i64 T = (i64)s[r] + o[r];
+        if (T <= Qp && o[r] <= Qo && mem + T <= M) { X.push_back(r); mem += T; }
+        else remaining.push_back(r);
+    }
+    std::stable_sort(remaining.begin(), remaining.end(), [&](int a, int b) {
+        __int128 l = (__int128)o[a] * ((i64)s[b] + o[b]), r = (__int128)o[b] * ((i64)s[a] + o[a]);
+        return l < r;
+    });
+    for (int r : remaining) {
+        i64 T = (i64)s[r] + o[r];
+        if (mem + T <= M) { X.push_back(r); mem += T; }
+    }
+    for (size_t k = 0; k < X.size(); ++k) chosen[k] = X[k];
+    return (int)X.size();
+}
+
+// The "random subset" of Algorithm 5, made reproducible: request id of batch number `batch` gets
+// the key mix(seed ^ mix(batch * 2^32 + id)) (splitmix64 finaliser); the sample is the
+// max(1, floor(m/2)) requests with the smallest keys, equal keys in the order of I (ascending o,
+// then index).  Writes the sample, returns its size.
+int orc_quantile_sample(int m, const int* ids, const int* o, uint64_t seed, int batch, int* sample) {
+    std::vector<int> I(ids, ids + m);
+    std::stable_sort(I.begin(), I.end(), [&](int a, int b) { if (o[a] != o[b]) return o[a] < o[b]; return a < b; });
+    std::vector<uint64_t> key(m);
+    std::vector<int> pos(m);
+    for (int k = 0; k < m; ++k) {
+        key[k] = mix64(seed ^ mix64(((uint64_t)(uint32_t)batch << 32) + (uint64_t)I[k]));
+        pos[k] = k;
+    }
+    std::stable_sort(pos.begin(), pos.end(), [&](int a, int b) { return key[a] < key[b]; });
+    int size = m / 2 > 1 ? m / 2 : 1;
+    for (int k = 0; k < size; ++k) sample[k] = I[pos[k]];
+    return size;
+}
+
+// Sorted-F with Algorithm 5 as the Phase-1 solver: repeat { sample; X = Algorithm 5 on the
+// remaining requests; sort X by (o, index); append }.
+int orc_sorted_f_quantile(int n, const int* s, const int* o, i64 M, uint64_t seed, int* order, int* batch_offsets) {
+    std::vector<int> rem(n);
+    std::iota(rem.begin(), rem.end(), 0);
+    std::vector<int> chosen(n), sample(n);
+    int pos = 0, nb = 0;
+    batch_offsets[0] = 0;
+    while (!rem.empty()) {
+        int ss = orc_quantile_sample((int)rem.size(), rem.data(), o, seed, nb, sample.data());
+        int c = orc_quantile_greedy_batch((int)rem.size(), rem.data(), s, o, M, ss, sample.data(), chosen.data(), 0, 0);
+        if (c <= 0) return -1;
+        std::vector<int> X(chosen.begin(), chosen.begin() + c);
         std::sort(X.begin(), X.end(), [&](int a, int b) { if (o[a] != o[b]) return o[a] < o[b]; return a < b; });
         std::vector<char> gone(n, 0);
         for (int x : X) { order[pos++] = x; gone[x] = 1; }

@@ -34,6 +34,16 @@ MUTATIONS = [
      "if (mem + dm >= M) continue;\n                i64 d_o", "test_local_swap_worked_by_hand", False),
     ("G-metric without the prefill term", "sw += a_num * s[r] + a_den * o[r];", "sw += a_den * o[r];",
      "test_sorted_g_reduces_to_f_and_differs_by_hand", False),
+    ("Algorithm 5 quantile position", "const int q = (int)((3ll * (sample_size - 1)) / 10);", "const int q = (int)((3ll * sample_size) / 10);",
+     "test_quantile_greedy_properties", False),
+    ("Algorithm 5 pass 2 stops at the first misfit", "for (int r : remaining) {\n        i64 T = (i64)s[r] + o[r];\n        if (mem + T <= M) { X.push_back(r); mem += T; }\n    }",
+     "for (int r : remaining) {\n        i64 T = (i64)s[r] + o[r];\n        if (mem + T <= M) { X.push_back(r); mem += T; } else break;\n    }",
+     "test_quantile_greedy_worked_by_hand", False),
+    ("Algorithm 5 ratio compared in floating point", "__int128 l = (__int128)o[a] * ((i64)s[b] + o[b]), r = (__int128)o[b] * ((i64)s[a] + o[a]);",
+     "double l = (double)o[a] / ((double)s[a] + o[a]), r = (double)o[b] / ((double)s[b] + o[b]);", "test_quantile_greedy_worked_by_hand", False),
+    ("Algorithm 5 without the output-length threshold", "if (T <= Qp && o[r] <= Qo && mem + T <= M)", "if (T <= Qp && mem + T <= M)",
+     "test_quantile_greedy_worked_by_hand", False),
+    ("Algorithm 5 sample of the wrong size", "int size = m / 2 > 1 ? m / 2 : 1;", "int size = (m + 1) / 2;", "test_quantile_greedy_properties", False),
     ("shortest-output-first sorts by size", "std::stable_sort(order, order + n, [&](int a, int b) { return o[a] < o[b]; });",
      "std::stable_sort(order, order + n, [&](int a, int b) { return s[a] + o[a] < s[b] + o[b]; });", "test_policies", False),
 ]

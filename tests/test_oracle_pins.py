@@ -506,3 +506,136 @@ def test_sorted_g_reduces_to_f_and_differs_by_hand():
     s, o = np.array([1, 1, 4], dtype=np.int32), np.array([4, 4, 1], dtype=np.int32)      # sizes 5, 5, 5; M = 10
     assert sorted(orc.sorted_f_local_swap(s, o, 10)[0][:2].tolist()) == [1, 2]           # F: o 1 < 4 -> swap request 0 out
     assert sorted(orc.sorted_g_local_swap(s, o, 10, 1, 1)[0][:2].tolist()) == [0, 1]     # G, alpha=1: weights 5,5,5 -> no swap
+
+
+# ---------------------------------------------------------------------------------------------
+# Algorithm 5 (Quantile Greedy Selection)
+# ---------------------------------------------------------------------------------------------
+def test_mix64_is_splitmix64():
+    # first three outputs of splitmix64 seeded with 0 (Steele, Lea, Flood; the generator's
+    # published reference values); mix64(z) is one step from state z
+    gamma = 0x9E3779B97F4A7C15
+    assert orc.mix64(0) == 0xE220A8397B1DCDAF
+    assert orc.mix64(gamma) == 0x6E789E6AA1B965F4
+    assert orc.mix64(2 * gamma) == 0x06C45D188009454F
+
+
+def test_quantile_greedy_worked_by_hand():
+    s = np.array([3, 5, 2, 8, 1, 4])
+    o = np.array([2, 1, 4, 3, 5, 2])
+    ids = np.arange(6)
+    # I by (o, index): 1, 0, 5, 3, 2, 4.  Sample {0,1,2}: s+o = 5,6,6 -> Q_p = 5 (position
+    # floor(0.3*2) = 0); o = 1,2,4 -> Q_o = 1.  Nothing passes both thresholds (request 1 has
+    # s+o = 6).  Ratios o/(s+o): r1 1/6, r3 3/11, r5 2/6, r0 2/5, r2 4/6, r4 5/6 -> first fit at
+    # M = 20 takes r1 (6), r3 (17) and nothing else.
+    X, qp, qo = orc.quantile_greedy_batch(ids, s, o, 20, [0, 1, 2])
+    assert (qp, qo) == (5, 1) and X.tolist() == [1, 3]
+    # Sample {0,1,3,5,2}: s+o = 5,6,6,6,11 -> Q_p = 6 (position floor(0.3*4) = 1); o = 1,2,2,3,4
+    # -> Q_o = 2.  Pass 1 admits r1, r0, r5 (mem 17).  Left over by ratio: r3, r2, r4.
+    X, qp, qo = orc.quantile_greedy_batch(ids, s, o, 18, [0, 1, 3, 5, 2])
+    assert (qp, qo) == (6, 2) and X.tolist() == [1, 0, 5]
+    # M = 23: pass 2 skips r3 (28 > 23) and goes on to admit r2 (23), then r4 no longer fits.
+    X, _, _ = orc.quantile_greedy_batch(ids, s, o, 23, [0, 1, 3, 5, 2])
+    assert X.tolist() == [1, 0, 5, 2]
+    # M = 15: r5 passes both thresholds but does not fit after r1 and r0; it falls to pass 2.
+    X, _, _ = orc.quantile_greedy_batch(ids, s, o, 15, [0, 1, 3, 5, 2])
+    assert X.tolist() == [1, 0]
+    # equal ratios (1/2 for both) keep the order of I; 1/3 < 333334/1000001 is decided exactly
+    # (thresholds (2, 1) from the sample {r2}: pass 1 takes r2 only; r1 then fills M = 10, r0 misfits)
+    X, _, _ = orc.quantile_greedy_batch([0, 1, 2], [4, 2, 1], [4, 2, 1], 10, [2])
+    assert X.tolist() == [2, 1]
+    # exact ratio comparison: with k = 2^28, r0 = (s k-1, o k) has ratio k/(2k-1) and r1 = (s k, o k+1)
+    # has (k+1)/(2k+1), smaller by 1/((2k-1)(2k+1)) ~ 2^-58 -- equal in double precision.  Pass 1
+    # takes r2 (thresholds (10, 1) from the sample {r2}); pass 2 must try r1 first, which then
+    # fills M = 10 + 2k+1 so that r0 misfits (a floating-point tie would admit r0 instead).
+    k = 1 << 28
+    X, _, _ = orc.quantile_greedy_batch([0, 1, 2], [k - 1, k, 9], [k, k + 1, 1], 10 + 2 * k + 1, [2])
+    assert X.tolist() == [2, 1]
+
+
+def test_quantile_greedy_properties():
+    rng = np.random.default_rng(77)
+    for trial in range(40):
+        n = int(rng.integers(1, 60))
+        M = int(rng.integers(20, 200))
+        s, o = random_instance(rng, n, M, M // 2, max(2, M // 4))
+        T = s + o
+        ids = rng.permutation(n)[: int(rng.integers(1, n + 1))]
+        sample = orc.quantile_sample(ids, o, 1234 + trial, trial)
+        m = len(ids)
+        assert len(sample) == max(1, m // 2) and len(set(sample.tolist())) == len(sample)
+        assert set(sample.tolist()) <= set(ids.tolist())
+        assert sample.tolist() == orc.quantile_sample(ids, o, 1234 + trial, trial).tolist()
+        X, qp, qo = orc.quantile_greedy_batch(ids, s, o, M, sample)
+        # thresholds against numpy's own lower quantile (element at floor(0.3 (m-1)))
+        if (3 * (len(sample) - 1)) % 10 != 0:        # away from the points where 0.3*(m-1) rounds in floating point
+            assert qp == int(np.quantile(T[sample], 0.3, method="lower"))
+            assert qo == int(np.quantile(o[sample], 0.3, method="lower"))
+        assert len(set(X.tolist())) == len(X) >= 1 and set(X.tolist()) <= set(ids.tolist())
+        mem = int(T[X].sum())
+        assert mem <= M
+        rest = [r for r in ids.tolist() if r not in set(X.tolist())]
+        assert all(mem + T[r] > M for r in rest)                 # first fit over everything: X is maximal
+        # the members that pass both thresholds come first, in ascending (o, index)
+        core = [r for r in X.tolist() if T[r] <= qp and o[r] <= qo]
+        k = 0
+        while k < len(X) and T[X[k]] <= qp and o[X[k]] <= qo:
+            k += 1
+        head = X[:k].tolist()
+        assert head == sorted(head, key=lambda r: (o[r], r))
+        # every request that passes both thresholds and is NOT in the head was refused for memory
+        # at its turn: the head members before it already fill M - T[r]
+        I = sorted(ids.tolist(), key=lambda r: (o[r], r))
+        mem1 = 0
+        for r in I:
+            if T[r] <= qp and o[r] <= qo:
+                if mem1 + T[r] <= M:
+                    assert r in head
+                    mem1 += T[r]
+        del core
+
+
+def test_quantile_sample_varies_with_seed_and_batch():
+    o = np.arange(1, 41)
+    ids = np.arange(40)
+    a = orc.quantile_sample(ids, o, 1, 0).tolist()
+    assert a != orc.quantile_sample(ids, o, 2, 0).tolist()
+    assert a != orc.quantile_sample(ids, o, 1, 1).tolist()
+    # the sample is the half with the smallest keys mix(seed ^ mix(batch * 2^32 + id))
+    keys = {i: orc.mix64(1 ^ orc.mix64((0 << 32) + i)) for i in range(40)}
+    assert sorted(a) == sorted(sorted(range(40), key=lambda i: keys[i])[:20])
+    # about half of all requests over many seeds: no request is favoured
+    hits = np.zeros(40)
+    for seed in range(400):
+        hits[orc.quantile_sample(ids, o, seed, 0)] += 1
+    assert hits.min() > 140 and hits.max() < 260
+
+
+def test_sorted_f_quantile_is_a_partition_into_feasible_maximal_batches():
+    rng = np.random.default_rng(78)
+    for trial in range(20):
+        n = int(rng.integers(1, 80))
+        M = int(rng.integers(20, 300))
+        s, o = random_instance(rng, n, M, M // 2, max(2, M // 4))
+        T = s + o
+        order, offs = orc.sorted_f_quantile(s, o, M, 99)
+        assert sorted(order.tolist()) == list(range(n))
+        assert offs[0] == 0 and offs[-1] == n and np.all(np.diff(offs) >= 1)
+        left = set(range(n))
+        for b in range(len(offs) - 1):
+            X = order[offs[b]: offs[b + 1]].tolist()
+            assert X == sorted(X, key=lambda r: (o[r], r))
+            mem = int(T[X].sum())
+            assert mem <= M
+            left -= set(X)
+            assert all(mem + T[r] > M for r in left)
+            # the batch is what the one-batch routine returns on the requests still there
+            rem = sorted(left | set(X))
+            sample = orc.quantile_sample(rem, o, 99, b)
+            Xb, _, _ = orc.quantile_greedy_batch(rem, s, o, M, sample)
+            assert sorted(Xb.tolist()) == sorted(X)
+    # Example 1 (Section 3): one request (s=63, o=1) and 21 requests (s=1, o=2), M = 64
+    s = np.array([63] + [1] * 21); o = np.array([1] + [2] * 21)
+    order, offs = orc.sorted_f_quantile(s, o, 64, 5)
+    tel = orc.list_schedule_alg1(s, o, 64, order)[1]
+    assert tel in (45, 64)                                     # one of the two batch orders the example discusses
