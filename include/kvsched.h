@@ -166,6 +166,21 @@ int sched_sorted_f_local_swap(sched_handle h, int32_t* order_out, int32_t* batch
 int sched_sorted_f_local_swap_dev(sched_handle h, int32_t* order_out, int32_t* batch_offsets_out,
                                   int32_t* num_batches_out, int64_t* tel_out);
 
+/* Sorted-F with Algorithm 5 (Quantile Greedy Selection, Section 5.3 and Appendix D) as the Phase-1
+ * solver: repeat on the requests not yet placed { walk them in ascending (o, index); draw a sample
+ * of max(1, floor(m/2)) of the m requests; Q_p, Q_o = 0.3-quantiles of s+o and of o over the sample;
+ * pass 1 admits, in walking order, every request with s+o <= Q_p, o <= Q_o that still fits in M;
+ * pass 2 walks the others in ascending o/(s+o) and admits every one that still fits; sort the batch
+ * by (o, index); append }.  What the listing leaves open is fixed as follows.  Sample: request id of
+ * batch number b (0-based) gets the key mix(seed ^ mix(b * 2^32 + id)), mix = one splitmix64 step;
+ * the sample is the requests with the smallest keys (equal keys in walking order).  Quantile: the
+ * element at 0-based position floor(3 (size-1) / 10) of the ascending values.  Ratios are compared
+ * exactly; equal ratios keep the walking order.
+ * SCHED_E_UNSUPPORTED when 2*bits(M) + bits(max o) > 63 (the exact ratio key would not fit 64 bits).
+ * Host pointers; synchronises once per batch; outputs and side effects as sched_sorted_f(). */
+int sched_sorted_f_quantile(sched_handle h, uint64_t seed, int32_t* order_out, int32_t* batch_offsets_out,
+                            int32_t* num_batches_out, int64_t* tel_out);
+
 /* Sorted-F with Algorithm 2 (exact dynamic programme, Section 5.1 and Appendix D) as the Phase-1
  * solver: repeat on the requests not yet placed { dp[k][m] = min sum of o over k-subsets whose
  * sum(s+o) is exactly m <= M, requests taken in ascending index, a cell replaced only by a strictly

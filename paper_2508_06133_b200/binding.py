@@ -22,7 +22,7 @@ NBHD_SWAP, NBHD_SWAP_INSERT, NBHD_SAMPLED = 0, 1, 2
 EXPORTS = [
     "sched_init", "sched_init_batch", "sched_set_stream", "sched_sync", "sched_set_prefill_weight", "sched_set_base_order",
     "sched_get_base_order", "sched_eval_batch", "sched_eval_batch_dev", "sched_sweep_dev",
-    "sched_sorted_f", "sched_sorted_f_dev", "sched_sorted_f_local_swap", "sched_sorted_f_local_swap_dev", "sched_sorted_f_dp", "sched_local_search", "sched_last_eval_kernel_ms", "sched_argmin_static_dev", "sched_stats", "sched_destroy",
+    "sched_sorted_f", "sched_sorted_f_dev", "sched_sorted_f_local_swap", "sched_sorted_f_local_swap_dev", "sched_sorted_f_dp", "sched_sorted_f_quantile", "sched_local_search", "sched_last_eval_kernel_ms", "sched_argmin_static_dev", "sched_stats", "sched_destroy",
     "sched_strerror", "sched_last_cuda_error",
 ]
 
@@ -67,6 +67,7 @@ def load():
     lib.sched_sorted_f_local_swap.argtypes = [vp, vp, vp, vp, vp]
     lib.sched_sorted_f_local_swap_dev.argtypes = [vp, vp, vp, vp, vp]
     lib.sched_sorted_f_dp.argtypes = [vp, vp, vp, vp, vp]
+    lib.sched_sorted_f_quantile.argtypes = [vp, C.c_uint64, vp, vp, vp, vp]
     lib.sched_local_search.argtypes = [vp, C.c_int, i32, u64, i64, vp, vp, vp, vp]
     lib.sched_stats.argtypes = [vp, vp, vp]
     lib.sched_last_eval_kernel_ms.argtypes = [vp, vp]
@@ -239,6 +240,16 @@ class Scheduler:
         nb, tel = C.c_int32(0), C.c_int64(0)
         _check(load().sched_sorted_f_dp(self._h, _np_ptr(order), _np_ptr(offs), C.byref(nb), C.byref(tel)),
                "sched_sorted_f_dp")
+        return order, offs[:nb.value + 1].copy(), tel.value
+
+    def sorted_f_quantile(self, seed=0):
+        """Sorted-F with Quantile Greedy Selection (Algorithm 5) as Phase-1 solver.
+        Returns (order, batch_offsets, TEL)."""
+        order = np.empty(self.n, dtype=np.int32)
+        offs = np.zeros(self.n + 1, dtype=np.int32)
+        nb, tel = C.c_int32(0), C.c_int64(0)
+        _check(load().sched_sorted_f_quantile(self._h, C.c_uint64(seed), _np_ptr(order), _np_ptr(offs), C.byref(nb), C.byref(tel)),
+               "sched_sorted_f_quantile")
         return order, offs[:nb.value + 1].copy(), tel.value
 
     def sorted_f_local_swap_dev(self, order_out=None, batch_offsets_out=None, num_batches_out=None, tel_out=None):

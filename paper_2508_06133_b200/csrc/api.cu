@@ -13,6 +13,7 @@
 #include "k2_fmetric.cuh"
 #include "k2_local_swap.cuh"
 #include "k2_dp.cuh"
+#include "k2_quantile.cuh"
 #include "k3_eval.cuh"
 #include "k5_argmin.cuh"
 
@@ -584,9 +585,10 @@ int sched_sweep_dev(sched_handle h, int sampled, uint64_t seed, int32_t iteratio
 }
 
 static int phase1_dp(sched_handle h);
+static int phase1_quantile(sched_handle h, u64 seed);
 
 static int sorted_f_common_dev(sched_handle h, int solver, int32_t* order_out, int32_t* batch_offsets_out,
-                               int32_t* num_batches_out, int64_t* tel_out) {
+                               int32_t* num_batches_out, int64_t* tel_out, u64 seed = 0) {
     KV_ENTER(h);
     if (h->batch_handle) return SCHED_E_INVAL;
     const int n = h->n;
@@ -604,9 +606,11 @@ static int sorted_f_common_dev(sched_handle h, int solver, int32_t* order_out, i
         KV_TRY(check_launch(h));
     } else if (solver == 2) {
         KV_TRY(phase1_dp(h));
+    } else if (solver == 3) {
+        KV_TRY(phase1_quantile(h, seed));
     } else {
         // Algorithm 4: ascending (s+o, index), then first fit + improving swaps, batch after batch
-        if (!h->d_ls) KV_TRY(dev_alloc(&h->d_ls, 7 * (size_t)n));
+        if (!h->d_ls) KV_TRY(dev_alloc(&h->d_ls, 7 * (size_t)n + 32));
         k1_keys_total_size<<<(n + 255) / 256, 256, 0, st>>>(h->d_s, h->d_o, n, h->d_keys_a, h->d_vals_a, SCHED_POLICY_TOTAL_SIZE);
         KV_TRY(check_launch(h));
         k1_radix_sort_segments<<<1, K1_THREADS, 0, st>>>(h->d_keys_a, h->d_vals_a, h->d_keys_b, h->d_vals_b, h->d_seg_off, nullptr, 1,
@@ -638,9 +642,9 @@ static int sorted_f_common_dev(sched_handle h, int solver, int32_t* order_out, i
 }
 
 static int sorted_f_common_host(sched_handle h, int solver, int32_t* order_out, int32_t* batch_offsets_out,
-                                int32_t* num_batches_out, int64_t* tel_out) {
+                                int32_t* num_batches_out, int64_t* tel_out, u64 seed = 0) {
     KV_ENTER(h);
-    KV_TRY(sorted_f_common_dev(h, solver, nullptr, nullptr, nullptr, nullptr));
+    KV_TRY(sorted_f_common_dev(h, solver, nullptr, nullptr, nullptr, nullptr, seed));
     const int n = h->n;
     cudaStream_t st = h->stream;
     int nb = 0;
@@ -718,6 +722,67 @@ static int phase1_dp(sched_handle h) {
     return rc;
 }
 
+// Algorithm 5 batch after batch; leaves the batches (members in ascending (o, index)) in d_vals_a and
+// the boundaries in d_batch_off / d_num_batches.  Reads the batch size back once per batch.
+static int phase1_quantile(sched_handle h, u64 seed) {
+    const int n = h->n;
+    cudaStream_t st = h->stream;
+    // fixed-point ratio key: 2^F must exceed the product of two sizes s+o <= M, and o * 2^F must fit
+    const int F = 2 * bits_of((u64)h->M);
+    if (F + bits_of((u64)h->omax) > 63) return SCHED_E_UNSUPPORTED;
+    if (!h->d_ls) KV_TRY(dev_alloc(&h->d_ls, 7 * (size_t)n + 32));
+    int* rem = h->d_ls;
+    int* rem_next = rem + n;
+    int* chosen = rem + 2 * (size_t)n;
+    int* va = rem + 3 * (size_t)n;
+    int* vb = rem + 4 * (size_t)n;
+    int* small = rem + 5 * (size_t)n + (n & 1);            // even offset: nothing here needs more
+    u64 *ka = h->d_keys_a, *kb = h->d_keys_b;
+    const int blocks = (n + 255) / 256;
+    // the remaining list: everything, ascending (o, index)
+    k1_keys_total_size<<<blocks, 256, 0, st>>>(h->d_s, h->d_o, n, ka, rem, SCHED_POLICY_SOF);
+    KV_TRY(check_launch(h));
+    k1_radix_sort_segments<<<1, K1_THREADS, 0, st>>>(ka, rem, kb, rem_next, h->d_seg_off, nullptr, 1,
+                                                      key_byte_mask(0, bits_of((u64)h->omax)));
+    KV_TRY(check_launch(h));
+    int zero = 0;
+    KV_CUDA(cudaMemcpyAsync(h->d_batch_off, &zero, sizeof(int), cudaMemcpyHostToDevice, st));
+    const unsigned mask_size = key_byte_mask(bits_of((u64)h->M), 0);
+    const unsigned mask_ratio = key_byte_mask(F + 1 < 32 ? F + 1 : 32, F + 1 > 32 ? F + 1 - 32 : 0) | 0x80u;
+    int nr = n, nb = 0, done = 0;
+    int* hp = (int*)h->h_pinned;
+    while (nr > 0) {
+        const int m = nr / 2 > 1 ? nr / 2 : 1;
+        const int g = (nr + 255) / 256;
+        k2q_begin<<<g, 256, 0, st>>>(rem, nr, seed, nb, ka, va, chosen, small);
+        KV_TRY(check_launch(h));
+        k1_radix_sort_segments<<<1, K1_THREADS, 0, st>>>(ka, va, kb, vb, small + K2Q_SEG1, nullptr, 1, 0xffu);
+        KV_TRY(check_launch(h));
+        k2q_sample_keys<<<(m + 255) / 256, 256, 0, st>>>(rem, va, m, h->d_s, h->d_o, ka);
+        KV_TRY(check_launch(h));
+        k1_radix_sort_segments<<<2, K1_THREADS, 0, st>>>(ka, va, kb, vb, small + K2Q_SEG2, nullptr, 2, mask_size);
+        KV_TRY(check_launch(h));
+        k2q_pass1<<<1, K2Q_THREADS, 0, st>>>(rem, nr, m, h->d_s, h->d_o, h->M, ka, chosen, small);
+        KV_TRY(check_launch(h));
+        k2q_ratio_keys<<<g, 256, 0, st>>>(rem, nr, h->d_s, h->d_o, chosen, F, ka, va);
+        KV_TRY(check_launch(h));
+        k1_radix_sort_segments<<<1, K1_THREADS, 0, st>>>(ka, va, kb, vb, small + K2Q_SEG1, nullptr, 1, mask_ratio);
+        KV_TRY(check_launch(h));
+        k2q_pass2_emit<<<1, K2Q_THREADS, 0, st>>>(rem, rem_next, nr, h->d_s, h->d_o, h->M, va, chosen, small,
+                                                  h->d_vals_a, done, h->d_batch_off, nb);
+        KV_TRY(check_launch(h));
+        KV_CUDA(cudaMemcpyAsync(hp, small + K2Q_COUNT, sizeof(int), cudaMemcpyDeviceToHost, st));
+        KV_CUDA(cudaStreamSynchronize(st));
+        const int took = *hp;
+        if (took < 1 || took > nr) return SCHED_E_INTERNAL;      // every batch places at least one request
+        nr -= took; done += took; ++nb;
+        int* tmp = rem; rem = rem_next; rem_next = tmp;
+    }
+    KV_CUDA(cudaMemcpyAsync(h->d_num_batches, &nb, sizeof(int), cudaMemcpyHostToDevice, st));
+    KV_CUDA(cudaStreamSynchronize(st));                          // nb lives on this stack frame
+    return SCHED_OK;
+}
+
 int sched_sorted_f_dev(sched_handle h, int32_t* order_out, int32_t* batch_offsets_out,
                        int32_t* num_batches_out, int64_t* tel_out) {
     return sorted_f_common_dev(h, 0, order_out, batch_offsets_out, num_batches_out, tel_out);
@@ -736,6 +801,11 @@ int sched_sorted_f_local_swap(sched_handle h, int32_t* order_out, int32_t* batch
 int sched_sorted_f_dp(sched_handle h, int32_t* order_out, int32_t* batch_offsets_out,
                       int32_t* num_batches_out, int64_t* tel_out) {
     return sorted_f_common_host(h, 2, order_out, batch_offsets_out, num_batches_out, tel_out);
+}
+
+int sched_sorted_f_quantile(sched_handle h, uint64_t seed, int32_t* order_out, int32_t* batch_offsets_out,
+                            int32_t* num_batches_out, int64_t* tel_out) {
+    return sorted_f_common_host(h, 3, order_out, batch_offsets_out, num_batches_out, tel_out, (u64)seed);
 }
 
 int sched_sorted_f(sched_handle h, int32_t* order_out, int32_t* batch_offsets_out,

@@ -234,6 +234,47 @@ def test_sorted_f_exact_dp_matches_oracle():
         assert e.value.code == kv.E_UNSUPPORTED
 
 
+def test_sorted_f_quantile_greedy_matches_oracle():
+    """Sorted-F with Algorithm 5 (Quantile Greedy Selection) as Phase-1 solver: batches, order, TEL."""
+    rng = np.random.default_rng(46)
+    cases = [W.tiny(), W.mixed_1k(), W.paper_scale(), W.mixed_10k()]
+    for trial in range(60):
+        n = int(rng.integers(1, 400))
+        M = int(rng.integers(10, 3000))
+        s, o = rand_instance(rng, n, M, M // 2, max(1, M // 3))
+        cases.append(W.Instance("rand", s, o, M))
+    # more than one 1024-position tile in both first-fit walks and in the hand-out
+    s, o = rand_instance(rng, 5000, 60000, 40, 30)
+    cases.append(W.Instance("many_small", s, o, 60000))
+    # many equal ratios and equal sizes: the stable orders decide
+    cases.append(W.Instance("ties", np.array([4, 4, 6, 8, 2, 3] * 40, dtype=np.int32), np.array([4, 6, 4, 2, 2, 3] * 40, dtype=np.int32), 90))
+    cases.append(W.Instance("ex1", np.array([63] + [1] * 21, dtype=np.int32), np.array([1] + [2] * 21, dtype=np.int32), 64))
+    cases.append(W.Instance("one", np.array([3], dtype=np.int32), np.array([2], dtype=np.int32), 5))
+    # ratios one part in 2^30 apart: r0 = k/(2k-1), r1 = (k+1)/(2k+1) with k = 2^14
+    k = 1 << 14
+    cases.append(W.Instance("close", np.array([k - 1, k, 9], dtype=np.int32), np.array([k, k + 1, 1], dtype=np.int32), 10 + 2 * k + 1))
+    for idx, inst in enumerate(cases):
+        seed = 1000 + idx
+        with kv.Scheduler(inst.s, inst.o, inst.M) as h:
+            order, offs, tel = h.sorted_f_quantile(seed)
+            assert (h.get_base_order() == order).all()
+        r_order, r_offs = orc.sorted_f_quantile(inst.s, inst.o, inst.M, seed)
+        assert (offs == r_offs).all(), inst.name
+        assert (order == r_order).all(), inst.name
+        assert tel == orc.list_schedule_rounds(inst.s, inst.o, inst.M, r_order)[1]
+    # a different seed draws different samples
+    inst = W.mixed_1k()
+    with kv.Scheduler(inst.s, inst.o, inst.M) as h:
+        a = h.sorted_f_quantile(1)[0]
+        b = h.sorted_f_quantile(2)[0]
+    assert (a != b).any()
+    # the exact ratio key needs 2 bits(M) + bits(max o) <= 63
+    with kv.Scheduler(np.array([5, 7], dtype=np.int32), np.array([512, 3], dtype=np.int32), 1 << 29) as h:
+        with pytest.raises(kv.SchedError) as e:
+            h.sorted_f_quantile(0)
+        assert e.value.code == kv.E_UNSUPPORTED
+
+
 def test_tiny_backlog_all_solvers_and_brute_force():
     """n = 16: prefix-F, Algorithm 4 and the exact DP orders, a full swap search from the DP order,
     and all 8! orders of the first 8 requests against the oracle's brute force."""
