@@ -18,6 +18,7 @@ _SO = os.path.join(_HERE, "liboracle.so")
 _lib = None
 
 FCFS, SHORTEST_OUTPUT_FIRST, TOTAL_SIZE_FIRST = 0, 1, 2
+SOF, SORTED_F = 1, 3                     # online policies: shortest decode first, Sorted-F-Online
 ENUM_ALG1, ENUM_SUM, DP = 0, 1, 2
 SWAP, SWAP_INSERT, SAMPLED = 0, 1, 2
 
@@ -280,3 +281,17 @@ def mix64(z):
     f = lib().orc_mix64
     f.restype = C.c_uint64
     return int(f(C.c_uint64(z & 0xFFFFFFFFFFFFFFFF)))
+
+
+def online_schedule(a, s, o, M, policy, period=10, lookahead=300):
+    """Online arrivals (FCFS, SOF recomputed every iteration, or Sorted-F-Online), iteration by
+    iteration.  Returns (start times, total latency = sum of p + o - a)."""
+    a, s, o = _i32(a), _i32(s), _i32(o)
+    n = len(s)
+    p = np.zeros(n, dtype=np.int64)
+    tot = C.c_longlong(0)
+    rc = lib().orc_online_schedule(n, _p(a), _p(s), _p(o), C.c_longlong(M), int(policy), int(period), int(lookahead),
+                                   p.ctypes.data_as(C.c_void_p), C.byref(tot))
+    if rc != 0:
+        raise ValueError("invalid online instance or parameters (%d)" % rc)
+    return p, tot.value

@@ -4,7 +4,8 @@
 // total end-to-end latency (Section 2.1-2.2, integer program of Section 6.1), the F-metric and
 // Sorted-F (Section 3, Algorithm 1), the exact dynamic programme (Section 5.1, Algorithm 2),
 // Local Swap Search and Quantile Greedy Selection (Sections 5.2-5.3, Algorithms 4 and 5),
-// Sorted-G (Section 7), and
+// Sorted-G (Section 7), the online policies of Section 6.3 (FCFS, shortest decode first and
+// Sorted-F-Online under arrivals over time), and
 // an order-level local search that scores every neighbour with Algorithm 1's Phase 2.  It exists
 // so that the GPU library can be checked against it; it shares no code with that library, is never
 // called by it, and nothing here is tuned for speed.  All arithmetic is integer.
@@ -738,6 +739,110 @@ int orc_sorted_f_quantile(int n, const int* s, const int* o, i64 M, uint64_t see
         rem.swap(rest);
     }
     return nb;
+}
+
+
+// ---------------------------------------------------------------------------------------------
+// O13. Online arrivals (Section 6.3 "Heuristics under Online Arrival", Section 7 "Experiment under
+//      Online Poisson Arrivals"), iteration by iteration.  Request i arrives at the integer time
+//      a_i >= 0 and may start at any p_i >= a_i, i.e. it is first seen by iteration a_i + 1 (with all
+//      a_i = 0 this is the offline model).  In every iteration t = 1, 2, ... the policy orders the
+//      pending requests (arrived, not started) and the executor admits the longest prefix of that
+//      order that fits the live memory profile -- Algorithm 1's Phase 2 step: walk the list, stop
+//      at the first request whose window [t, t+o) would exceed M in some round.
+//        policy 0  FCFS: arrival (index) order.
+//        policy 1  shortest decode first, recomputed every iteration: ascending (o, index).
+//        policy 3  Sorted-F-Online: a cached priority list; requests that arrive are appended to it;
+//                  it is recomputed when it has never been computed, when `period` iterations have
+//                  passed since the last recomputation, when the cached list had run empty, or when
+//                  the arrivals since the last recomputation reach half of the backlog size at that
+//                  recomputation.  Recomputation: sort the pending requests by ascending
+//                  (s+o, index); the first `lookahead` of them are ordered by Sorted-F with
+//                  Algorithm 4 (batch after batch, each batch by ascending (o, index)), the others
+//                  follow in the (s+o, index) order.
+//      Left open by the text and fixed here: integer arrival times and "seen from iteration a+1";
+//      which pending requests form the look-ahead window (the first `lookahead` in the fallback
+//      order); arrivals between recomputations go to the tail in index order; a recomputation is
+//      only considered while something is pending.
+// Writes the start times, returns 0; total_latency (nullable) = sum of (p_i + o_i - a_i).
+// ---------------------------------------------------------------------------------------------
+static void online_recompute(std::vector<int>& cached, const int* s, const int* o, i64 M, int lookahead) {
+    std::vector<int> P(cached);
+    std::sort(P.begin(), P.end(), [&](int x, int y) {
+        int tx = s[x] + o[x], ty = s[y] + o[y];
+        if (tx != ty) return tx < ty;
+        return x < y;
+    });
+    const int m = (int)P.size();
+    const int wn = m < lookahead ? m : lookahead;
+    std::vector<int> win(P.begin(), P.begin() + wn), out, chosen(wn > 0 ? wn : 1);
+    while (!win.empty()) {
+        int c = orc_local_swap_batch((int)win.size(), win.data(), s, o, M, chosen.data(), 0);
+        std::vector<int> X(chosen.begin(), chosen.begin() + c);
+        std::sort(X.begin(), X.end(), [&](int x, int y) { if (o[x] != o[y]) return o[x] < o[y]; return x < y; });
+        for (int x : X) out.push_back(x);
+        std::vector<int> rest;
+        for (int r : win) if (std::find(X.begin(), X.end(), r) == X.end()) rest.push_back(r);
+        win.swap(rest);
+    }
+    for (int k = wn; k < m; ++k) out.push_back(P[k]);
+    cached.swap(out);
+}
+
+int orc_online_schedule(int n, const int* a, const int* s, const int* o, i64 M, int policy,
+                        int period, int lookahead, i64* p_out, i64* total_latency) {
+    if (n <= 0 || period < 1 || lookahead < 1) return -1;
+    if (policy != 0 && policy != 1 && policy != 3) return -1;
+    i64 horizon = 2;
+    for (int i = 0; i < n; ++i) {
+        if (a[i] < 0 || s[i] < 1 || o[i] < 1 || (i64)s[i] + o[i] > M) return -1;
+        horizon = std::max<i64>(horizon, a[i]);
+    }
+    for (int i = 0; i < n; ++i) horizon += o[i];
+    std::vector<i64> U((size_t)horizon + 2, 0);          // U[tau]: memory in use in round tau
+    std::vector<char> started(n, 0), seen(n, 0);
+    std::vector<int> cached;                              // policy 3: the priority list
+    bool computed = false;
+    i64 t_last = 0, backlog_last = 0, new_since = 0;
+    int remaining = n;
+    for (i64 t = 1; remaining > 0; ++t) {
+        if (t > horizon + 1) return -2;                   // cannot happen: by then everything fits
+        std::vector<int> newly;
+        for (int i = 0; i < n; ++i) if (!seen[i] && a[i] <= t - 1) { seen[i] = 1; newly.push_back(i); }
+        std::vector<int> list;
+        if (policy == 3) {
+            const bool was_empty = cached.empty();
+            for (int i : newly) cached.push_back(i);
+            new_since += (i64)newly.size();
+            if (!cached.empty()) {
+                if (!computed || t - t_last >= period || was_empty || 2 * new_since >= backlog_last) {
+                    online_recompute(cached, s, o, M, lookahead);
+                    computed = true; t_last = t; backlog_last = (i64)cached.size(); new_since = 0;
+                }
+            }
+            list = cached;
+        } else {
+            for (int i = 0; i < n; ++i) if (seen[i] && !started[i]) list.push_back(i);
+            if (policy == 1)
+                std::stable_sort(list.begin(), list.end(), [&](int x, int y) { return o[x] < o[y]; });
+        }
+        size_t taken = 0;
+        for (int r : list) {
+            bool fits = true;
+            for (int j = 1; j <= o[r]; ++j)
+                if (U[t - 1 + j] + s[r] + j > M) { fits = false; break; }
+            if (!fits) break;
+            for (int j = 1; j <= o[r]; ++j) U[t - 1 + j] += (i64)s[r] + j;
+            p_out[r] = t - 1; started[r] = 1; --remaining; ++taken;
+        }
+        if (policy == 3) cached.erase(cached.begin(), cached.begin() + taken);
+    }
+    if (total_latency) {
+        i64 tot = 0;
+        for (int i = 0; i < n; ++i) tot += p_out[i] + o[i] - a[i];
+        *total_latency = tot;
+    }
+    return 0;
 }
 
 }  // extern "C"

@@ -160,3 +160,39 @@ def random_permutations(n: int, count: int, seed: int) -> np.ndarray:
     for c in range(count):
         out[c] = np.argsort(u64(seed, 100 + c, k), kind="stable").astype(np.int32)
     return out
+
+
+@dataclass(frozen=True)
+class OnlineInstance:
+    name: str
+    a: np.ndarray          # int32 [n]   arrival times, non-decreasing
+    s: np.ndarray          # int32 [n]
+    o: np.ndarray          # int32 [n]
+    M: int
+
+    @property
+    def n(self) -> int:
+        return int(self.s.shape[0])
+
+
+def online_poisson(lam: float, horizon: int = 4000, seed: int = 11, M: int = 16492) -> OnlineInstance:
+    """Poisson arrivals of rate ``lam`` per iteration over ``horizon`` iterations (Section 7, online
+    experiment): exponential gaps from the counter-based generator, arrival time = floor of the
+    running sum, arrivals at or after ``horizon`` dropped; lengths as in ``paper_scale``."""
+    kmax = int(lam * horizon * 1.5 + 64)
+    k = np.arange(kmax)
+    gaps = -np.log(1.0 - uniform01(seed, 40, k)) / lam
+    times = np.floor(np.cumsum(gaps)).astype(np.int64)
+    n = int(np.searchsorted(times, horizon, side="left"))
+    n = max(n, 1)
+    base = paper_scale(seed=seed, n=kmax)
+    return OnlineInstance("online_lam%.2f_seed%d" % (lam, seed), times[:n].astype(np.int32),
+                          base.s[:n].copy(), base.o[:n].copy(), M)
+
+
+def memory_bound_rate(s: np.ndarray, o: np.ndarray, M: int) -> float:
+    """Arrival rate at which the mean KV-memory demand per iteration equals M: a request holds
+    s + j tokens in its j-th round, so it needs sum_j (s + j) token-rounds."""
+    s = s.astype(np.float64)
+    o = o.astype(np.float64)
+    return float(M / np.mean(o * s + o * (o + 1) / 2))

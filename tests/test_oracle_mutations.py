@@ -44,6 +44,15 @@ MUTATIONS = [
     ("Algorithm 5 without the output-length threshold", "if (T <= Qp && o[r] <= Qo && mem + T <= M)", "if (T <= Qp && mem + T <= M)",
      "test_quantile_greedy_worked_by_hand", False),
     ("Algorithm 5 sample of the wrong size", "int size = m / 2 > 1 ? m / 2 : 1;", "int size = (m + 1) / 2;", "test_quantile_greedy_properties", False),
+    ("online: early refresh at 100 % instead of 50 %", "|| 2 * new_since >= backlog_last) {", "|| new_since >= backlog_last) {",
+     "test_sorted_f_online_worked_by_hand", False),
+    ("online: a refused head is skipped", "if (!fits) break;\n            for (int j = 1; j <= o[r]; ++j) U[t - 1 + j] += (i64)s[r] + j;",
+     "if (!fits) continue;\n            for (int j = 1; j <= o[r]; ++j) U[t - 1 + j] += (i64)s[r] + j;", "test_online_fcfs_and_shortest_first_worked_by_hand", False),
+    ("online: arrivals seen one iteration early", "if (!seen[i] && a[i] <= t - 1)", "if (!seen[i] && a[i] <= t)",
+     "test_online_underloaded_requests_start_on_arrival", False),
+    ("online: no look-ahead cap", "const int wn = m < lookahead ? m : lookahead;", "const int wn = m;", "test_sorted_f_online_worked_by_hand", False),
+    ("online: periodic refresh never fires", "if (!computed || t - t_last >= period || was_empty", "if (!computed || was_empty",
+     "test_sorted_f_online_worked_by_hand", False),
     ("shortest-output-first sorts by size", "std::stable_sort(order, order + n, [&](int a, int b) { return o[a] < o[b]; });",
      "std::stable_sort(order, order + n, [&](int a, int b) { return s[a] + o[a] < s[b] + o[b]; });", "test_policies", False),
 ]

@@ -639,3 +639,120 @@ def test_sorted_f_quantile_is_a_partition_into_feasible_maximal_batches():
     order, offs = orc.sorted_f_quantile(s, o, 64, 5)
     tel = orc.list_schedule_alg1(s, o, 64, order)[1]
     assert tel in (45, 64)                                     # one of the two batch orders the example discusses
+
+
+# ---------------------------------------------------------------------------------------------
+# Online arrivals (Section 6.3, Section 7's Poisson experiment)
+# ---------------------------------------------------------------------------------------------
+ONLINE_POLICIES = (orc.FCFS, orc.SOF, orc.SORTED_F)
+
+
+def test_online_with_everything_present_at_time_zero_is_the_offline_model():
+    rng = np.random.default_rng(91)
+    for trial in range(12):
+        n = int(rng.integers(1, 40))
+        M = int(rng.integers(20, 200))
+        s, o = random_instance(rng, n, M, M // 2, max(2, M // 4))
+        a = np.zeros(n, dtype=np.int32)
+        for pol in (orc.FCFS, orc.SOF):
+            p, tot = orc.online_schedule(a, s, o, M, pol)
+            rp, rtel, _ = orc.list_schedule_alg1(s, o, M, orc.policy_order(s, o, pol))
+            assert (p == rp).all() and tot == rtel
+        # one planning pass over the whole backlog, never repeated: Sorted-F with Algorithm 4
+        p, tot = orc.online_schedule(a, s, o, M, orc.SORTED_F, period=1 << 30, lookahead=n)
+        order = orc.sorted_f_local_swap(s, o, M)[0]
+        rp, rtel, _ = orc.list_schedule_alg1(s, o, M, order)
+        assert (p == rp).all() and tot == rtel
+
+
+def test_online_underloaded_requests_start_on_arrival():
+    rng = np.random.default_rng(92)
+    n, M = 30, 100
+    s, o = random_instance(rng, n, M, 50, 20)
+    a = np.cumsum(rng.integers(21, 40, n)).astype(np.int32)        # gaps longer than any decode
+    for pol in ONLINE_POLICIES:
+        p, tot = orc.online_schedule(a, s, o, M, pol)
+        assert (p == a).all() and tot == int(o.sum())
+
+
+def test_online_schedules_are_feasible_and_fcfs_is_earliest_fit_in_arrival_order():
+    rng = np.random.default_rng(93)
+    for trial in range(10):
+        n = int(rng.integers(2, 50))
+        M = int(rng.integers(20, 120))
+        s, o = random_instance(rng, n, M, M // 2, max(2, M // 4))
+        a = np.sort(rng.integers(0, 3 * n, n)).astype(np.int32)
+        for pol in ONLINE_POLICIES:
+            p, tot = orc.online_schedule(a, s, o, M, pol, period=int(rng.integers(1, 6)), lookahead=int(rng.integers(1, 12)))
+            assert (p >= a).all()
+            chk = orc.check_schedule(s, o, M, p)
+            assert chk["feasible"] and chk["peak"] <= M and tot == chk["tel"] - int(a.sum())
+        # FCFS by its definition: request i starts at the first p >= max(a_i, p_{i-1}) at which
+        # every round of its stay is within M, given the earlier requests
+        p, _ = orc.online_schedule(a, s, o, M, orc.FCFS)
+        U = np.zeros(int(a.max()) + int(o.sum()) + 2, dtype=np.int64)
+        prev = 0
+        for i in range(n):
+            q = max(int(a[i]), prev)
+            while any(U[q + j] + s[i] + j > M for j in range(1, o[i] + 1)):
+                q += 1
+            assert p[i] == q
+            for j in range(1, o[i] + 1):
+                U[q + j] += s[i] + j
+            prev = q
+
+
+def test_online_fcfs_and_shortest_first_worked_by_hand():
+    # M = 10; r0 (a 0, s 4, o 3), r1 (a 0, s 5, o 4), r2 (a 1, s 2, o 1).
+    a, s, o = [0, 0, 1], [4, 5, 2], [3, 4, 1]
+    # FCFS: iteration 1 admits r0 (rounds 1-3 use 5,6,7); r1 would make round 1 use 11.  r1 stays
+    # at the head and is refused in iterations 2 and 3 (rounds 2, 3 still hold 6, 7), which also
+    # holds r2 back; iteration 4 admits r1 (p = 3) and then r2 (round 4: 6 + 3 = 9).
+    p, tot = orc.online_schedule(a, s, o, 10, orc.FCFS)
+    assert p.tolist() == [0, 3, 3] and tot == 3 + 7 + 3
+    # shortest first: in iteration 2 r2 (o = 1) goes ahead of r1 and fits (round 2: 6 + 3 = 9).
+    p, tot = orc.online_schedule(a, s, o, 10, orc.SOF)
+    assert p.tolist() == [0, 3, 1] and tot == 3 + 7 + 1
+
+
+def test_sorted_f_online_worked_by_hand():
+    M = 10
+    # Example A (period 3, look-ahead 2): r0, r1 = (a 0, s 1, o 2), r2 = (0, 6, 1), r3 = (1, 1, 1),
+    # r4 = (2, 2, 1), r5 = (6, 3, 2).
+    #  it 1: first plan.  By (s+o, index): r0, r1 | r2 -- only the first two are planned: one batch
+    #        {r0, r1}; list r0, r1, r2.  r0, r1 start (round 1 holds 4, round 2 holds 6); r2 would
+    #        make round 1 hold 11.
+    #  it 2: r3 arrives, goes to the tail (1 arrival < half of 3).  r2 refused (round 2: 6 + 7);
+    #        r3 waits behind it.
+    #  it 3: r4 arrives: 2 arrivals >= half of 3 -> new plan: r3, r4 | r2 -> list r3, r4, r2.
+    #        r3 and r4 start (round 3 holds 5); r2 refused (12).
+    #  it 4: r2 starts.  it 7: r5 has arrived, the list had run empty -> plan; r5 starts.
+    a, s, o = [0, 0, 0, 1, 2, 6], [1, 1, 6, 1, 2, 3], [2, 2, 1, 1, 1, 2]
+    p, tot = orc.online_schedule(a, s, o, M, orc.SORTED_F, period=3, lookahead=2)
+    assert p.tolist() == [0, 0, 3, 2, 2, 6] and tot == 2 + 2 + 4 + 2 + 1 + 2
+    # with a look-ahead of 3 the first plan swaps r0 out for r2 (o 1 < 2, memory 3+7 = 10 fits):
+    # batch {r2, r1}, then {r0}
+    p3, _ = orc.online_schedule(a, s, o, M, orc.SORTED_F, period=3, lookahead=3)
+    assert p3[2] == 0 and p3[1] == 0 and p3[0] > 0
+    # Example B (look-ahead 10): r0 = (0, 5, 4), r1 = (0, 6, 3), r2 = (0, 6, 2), r3 = (0, 7, 2),
+    # r4 = (1, 1, 1).  First plan: batches {r2}, {r3}, {r1}, {r0} (each is alone: two never fit;
+    # Algorithm 4 walks to the shortest decode).  r2 starts in iteration 1; r3 is refused in
+    # iterations 1 and 2 (rounds 1, 2 hold 7, 8); r4 arrives in iteration 2 and waits at the tail
+    # although it would fit (8 + 2).
+    a, s, o = [0, 0, 0, 0, 1], [5, 6, 6, 7, 1], [4, 3, 2, 2, 1]
+    #  period 2: iteration 3 plans again: by size r4 first -> list r4, r3, r1, r0; r4 and r3 start
+    #  (round 3: 2 + 8 = 10), r1 in iteration 5, r0 in iteration 8.
+    p, tot = orc.online_schedule(a, s, o, M, orc.SORTED_F, period=2, lookahead=10)
+    assert p.tolist() == [7, 4, 0, 2, 2] and tot == 11 + 7 + 2 + 4 + 2
+    #  period 100: no new plan (1 arrival < half of 4): r4 stays last and starts with r0 in iteration 8.
+    p, _ = orc.online_schedule(a, s, o, M, orc.SORTED_F, period=100, lookahead=10)
+    assert p.tolist() == [7, 4, 0, 2, 7]
+
+
+def test_online_overload_ranking_of_the_three_policies():
+    # Section 7, online experiment: under overload Sorted-F-Online has the lowest mean latency and
+    # FCFS by far the highest (the paper: 15-40 % below shortest-decode-first, 83-88 % below FCFS)
+    inst = W.online_poisson(0.25, horizon=1500, seed=3)
+    lat = {pol: orc.online_schedule(inst.a, inst.s, inst.o, inst.M, pol)[1] for pol in ONLINE_POLICIES}
+    assert lat[orc.SORTED_F] < lat[orc.SOF] < lat[orc.FCFS]
+    assert lat[orc.SORTED_F] < 0.5 * lat[orc.FCFS]
