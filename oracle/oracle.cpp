@@ -4,7 +4,7 @@
 // total end-to-end latency (Section 2.1-2.2, integer program of Section 6.1), the F-metric and
 // Sorted-F (Section 3, Algorithm 1), the exact dynamic programme (Section 5.1, Algorithm 2),
 // Local Swap Search and Quantile Greedy Selection (Sections 5.2-5.3, Algorithms 4 and 5),
-// Sorted-G (Section 7), the online policies of Section 6.3 (FCFS, shortest decode first and
+// Sorted-G (Section 7), the online policies of Section 6.2 (FCFS, shortest decode first and
 // Sorted-F-Online under arrivals over time), and
 // an order-level local search that scores every neighbour with Algorithm 1's Phase 2.  It exists
 // so that the GPU library can be checked against it; it shares no code with that library, is never
@@ -743,7 +743,7 @@ int orc_sorted_f_quantile(int n, const int* s, const int* o, i64 M, uint64_t see
 
 
 // ---------------------------------------------------------------------------------------------
-// O13. Online arrivals (Section 6.3 "Heuristics under Online Arrival", Section 7 "Experiment under
+// O13. Online arrivals (Section 6.2 "Heuristics under Online Arrival", Section 7 "Experiment under
 //      Online Poisson Arrivals"), iteration by iteration.  Request i arrives at the integer time
 //      a_i >= 0 and may start at any p_i >= a_i, i.e. it is first seen by iteration a_i + 1 (with all
 //      a_i = 0 this is the offline model).  In every iteration t = 1, 2, ... the policy orders the

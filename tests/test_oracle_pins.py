@@ -642,7 +642,7 @@ def test_sorted_f_quantile_is_a_partition_into_feasible_maximal_batches():
 
 
 # ---------------------------------------------------------------------------------------------
-# Online arrivals (Section 6.3, Section 7's Poisson experiment)
+# Online arrivals (Section 6.2, Section 7's Poisson experiment)
 # ---------------------------------------------------------------------------------------------
 ONLINE_POLICIES = (orc.FCFS, orc.SOF, orc.SORTED_F)
 
