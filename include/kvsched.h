@@ -233,6 +233,32 @@ int sched_last_eval_kernel_ms(sched_handle h, float* ms_out);
 int sched_argmin_static_dev(const int64_t* tel, int64_t count, int64_t index_base,
                             int64_t* best_out, void* cuda_stream);
 
+/* Online arrivals (Section 6.2, "Heuristics under Online Arrival"; Section 7's Poisson experiment):
+ * B independent arrival streams simulated to completion under one policy, one CTA per stream.
+ * Stream b has n_each[b] <= n_max requests in row b of the [B, n_max] arrays arrival / s / o (row
+ * entries past n_each[b] are ignored).  Request i arrives at the integer time arrival[i] >= 0
+ * (non-decreasing within a row), may start at any p >= arrival[i] (it is first seen by iteration
+ * arrival[i] + 1) and then occupies rounds p+1 .. p+o exactly as in the offline model.  In every
+ * iteration the policy orders the pending requests and the longest prefix of that order that fits
+ * the live memory profile is admitted (Algorithm 1, Phase 2).
+ *   SCHED_POLICY_FCFS      arrival order.
+ *   SCHED_POLICY_SOF       ascending (o, index), recomputed every iteration.
+ *   SCHED_POLICY_SORTED_F  Sorted-F-Online: a cached priority list; arrivals are appended to it; it is
+ *       planned again when it has never been planned, `period` iterations after the last plan, when
+ *       it had run empty, or when the arrivals since the last plan reach half of the backlog size at
+ *       that plan.  A plan sorts the pending requests by ascending (s+o, index), orders the first
+ *       `lookahead` of them by Sorted-F with Algorithm 4 (every batch by ascending (o, index)) and
+ *       appends the others in sorted order.  The paper uses period = 10, lookahead = 300.
+ * start_out [B, n_max] receives the start times (-1 where a row has no request), latency_out [B] the
+ * sum of (p + o - arrival) per stream; kernel_ms_out (nullable) the device time of the simulation.
+ * All pointers are host memory; the call allocates and frees its own device buffers and
+ * synchronises the device.  SCHED_E_INVAL: bad sizes, policy, period or lookahead < 1, a request with
+ * s < 1, o < 1 or s+o > M, decreasing arrivals.  SCHED_E_UNSUPPORTED: n_max > 2048, lookahead > 1024,
+ * o > 8192, M >= 2^30, arrival >= 2^29, or a stream whose decode lengths sum to 2^29 or more. */
+int sched_online_simulate(int32_t B, int32_t n_max, const int32_t* n_each, const int32_t* arrival,
+                          const int32_t* s, const int32_t* o, int64_t M, int32_t policy, int32_t period,
+                          int32_t lookahead, int32_t* start_out, int64_t* latency_out, float* kernel_ms_out);
+
 /* Counters since sched_init: kernels launched by this handle, candidates evaluated. */
 int sched_stats(sched_handle h, int64_t* kernel_launches_out, int64_t* evaluations_out);
 

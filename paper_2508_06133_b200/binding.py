@@ -22,7 +22,7 @@ NBHD_SWAP, NBHD_SWAP_INSERT, NBHD_SAMPLED = 0, 1, 2
 EXPORTS = [
     "sched_init", "sched_init_batch", "sched_set_stream", "sched_sync", "sched_set_prefill_weight", "sched_set_base_order",
     "sched_get_base_order", "sched_eval_batch", "sched_eval_batch_dev", "sched_sweep_dev",
-    "sched_sorted_f", "sched_sorted_f_dev", "sched_sorted_f_local_swap", "sched_sorted_f_local_swap_dev", "sched_sorted_f_dp", "sched_sorted_f_quantile", "sched_local_search", "sched_last_eval_kernel_ms", "sched_argmin_static_dev", "sched_stats", "sched_destroy",
+    "sched_sorted_f", "sched_sorted_f_dev", "sched_sorted_f_local_swap", "sched_sorted_f_local_swap_dev", "sched_sorted_f_dp", "sched_sorted_f_quantile", "sched_online_simulate", "sched_local_search", "sched_last_eval_kernel_ms", "sched_argmin_static_dev", "sched_stats", "sched_destroy",
     "sched_strerror", "sched_last_cuda_error",
 ]
 
@@ -68,6 +68,7 @@ def load():
     lib.sched_sorted_f_local_swap_dev.argtypes = [vp, vp, vp, vp, vp]
     lib.sched_sorted_f_dp.argtypes = [vp, vp, vp, vp, vp]
     lib.sched_sorted_f_quantile.argtypes = [vp, C.c_uint64, vp, vp, vp, vp]
+    lib.sched_online_simulate.argtypes = [i32, i32, vp, vp, vp, vp, i64, i32, i32, i32, vp, vp, vp]
     lib.sched_local_search.argtypes = [vp, C.c_int, i32, u64, i64, vp, vp, vp, vp]
     lib.sched_stats.argtypes = [vp, vp, vp]
     lib.sched_last_eval_kernel_ms.argtypes = [vp, vp]
@@ -281,3 +282,22 @@ def argmin_static_dev(tel, best_out, *, count=None, index_base=0, stream=None):
     ptr = C.c_void_p(stream.cuda_stream) if stream is not None else None
     _check(load().sched_argmin_static_dev(_dev_ptr(tel), n, index_base, _dev_ptr(best_out), ptr),
            "sched_argmin_static_dev")
+
+
+def online_simulate(n_each, arrival, s, o, M, policy, period=10, lookahead=300):
+    """B arrival streams under one online policy (rows of [B, n_max] arrays; see sched_online_simulate).
+    Returns (start times [B, n_max], total latency per stream [B], kernel milliseconds)."""
+    arrival = np.ascontiguousarray(arrival, dtype=np.int32)
+    s = np.ascontiguousarray(s, dtype=np.int32)
+    o = np.ascontiguousarray(o, dtype=np.int32)
+    n_each = np.ascontiguousarray(n_each, dtype=np.int32)
+    if arrival.ndim != 2 or s.shape != arrival.shape or o.shape != arrival.shape or n_each.shape != (arrival.shape[0],):
+        raise ValueError("arrival, s, o must be [B, n_max] and n_each [B]")
+    B, n_max = arrival.shape
+    starts = np.empty((B, n_max), dtype=np.int32)
+    lat = np.empty(B, dtype=np.int64)
+    ms = C.c_float(0.0)
+    _check(load().sched_online_simulate(B, n_max, _np_ptr(n_each), _np_ptr(arrival), _np_ptr(s), _np_ptr(o), int(M),
+                                        int(policy), int(period), int(lookahead), _np_ptr(starts), _np_ptr(lat), C.byref(ms)),
+           "sched_online_simulate")
+    return starts, lat, ms.value

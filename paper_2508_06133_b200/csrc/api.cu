@@ -16,6 +16,7 @@
 #include "k2_quantile.cuh"
 #include "k3_eval.cuh"
 #include "k5_argmin.cuh"
+#include "k6_online.cuh"
 
 thread_local char g_last_cuda_error[256] = "";
 
@@ -874,6 +875,87 @@ int sched_last_eval_kernel_ms(sched_handle h, float* ms_out) {
     KV_CUDA(cudaEventSynchronize(h->ev_k3_end));
     KV_CUDA(cudaEventElapsedTime(ms_out, h->ev_k3_begin, h->ev_k3_end));
     return SCHED_OK;
+}
+
+int sched_online_simulate(int32_t B, int32_t n_max, const int32_t* n_each, const int32_t* arrival,
+                          const int32_t* s, const int32_t* o, int64_t M, int32_t policy, int32_t period,
+                          int32_t lookahead, int32_t* start_out, int64_t* latency_out, float* kernel_ms_out) {
+    if (B < 1 || n_max < 1 || n_max > K6_MAX_N || !n_each || !arrival || !s || !o || !start_out || !latency_out)
+        return SCHED_E_INVAL;
+    if (policy != SCHED_POLICY_FCFS && policy != SCHED_POLICY_SOF && policy != SCHED_POLICY_SORTED_F) return SCHED_E_INVAL;
+    if (period < 1 || lookahead < 1 || M < 2) return SCHED_E_INVAL;
+    if (M >= (1ll << 30) || lookahead > K6_MAX_LOOKAHEAD) return SCHED_E_UNSUPPORTED;
+    int omax = 1;
+    for (int b = 0; b < B; ++b) {
+        const int n = n_each[b];
+        if (n < 1 || n > n_max) return SCHED_E_INVAL;
+        const size_t base = (size_t)b * n_max;
+        i64 sum_o = 0;
+        for (int i = 0; i < n; ++i) {
+            const int ai = arrival[base + i], si = s[base + i], oi = o[base + i];
+            if (ai < 0 || si < 1 || oi < 1 || (i64)si + oi > M) return SCHED_E_INVAL;
+            if (i > 0 && ai < arrival[base + i - 1]) return SCHED_E_INVAL;
+            if (ai >= (1 << 29)) return SCHED_E_UNSUPPORTED;
+            omax = oi > omax ? oi : omax;
+            sum_o += oi;
+        }
+        if (sum_o >= (1ll << 29)) return SCHED_E_UNSUPPORTED;
+    }
+    if (omax > K6_MAX_O) return SCHED_E_UNSUPPORTED;
+    OnlineParams P;
+    memset(&P, 0, sizeof(P));
+    P.n_max = n_max; P.M = (int)M; P.policy = policy; P.period = period; P.lookahead = lookahead;
+    P.L = 32; while (P.L < omax) P.L <<= 1;
+    P.npow2 = 2; while (P.npow2 < n_max) P.npow2 <<= 1;
+    const size_t smem = sizeof(u64) * (size_t)P.npow2 + sizeof(int) * ((size_t)5 * n_max + P.L + (size_t)9 * lookahead);
+    int dev = 0, optin = 0;
+    KV_CUDA(cudaGetDevice(&dev));
+    KV_CUDA(cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+    if (smem + 4096 > (size_t)optin) return SCHED_E_UNSUPPORTED;
+    KV_CUDA(cudaFuncSetAttribute(k6_online, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+
+    const size_t cells = (size_t)B * n_max;
+    int *d_n = nullptr, *d_a = nullptr, *d_s = nullptr, *d_o = nullptr, *d_start = nullptr, *d_status = nullptr;
+    i64* d_lat = nullptr;
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    int rc = SCHED_OK;
+    do {
+#define ON_CUDA(call) if ((call) != cudaSuccess) { rc = kv_cuda_fail(cudaGetLastError(), #call); break; }
+        if ((rc = dev_alloc(&d_n, (size_t)B)) != SCHED_OK) break;
+        if ((rc = dev_alloc(&d_a, cells)) != SCHED_OK) break;
+        if ((rc = dev_alloc(&d_s, cells)) != SCHED_OK) break;
+        if ((rc = dev_alloc(&d_o, cells)) != SCHED_OK) break;
+        if ((rc = dev_alloc(&d_start, cells)) != SCHED_OK) break;
+        if ((rc = dev_alloc(&d_lat, (size_t)B)) != SCHED_OK) break;
+        if ((rc = dev_alloc(&d_status, 1)) != SCHED_OK) break;
+        ON_CUDA(cudaEventCreate(&e0));
+        ON_CUDA(cudaEventCreate(&e1));
+        ON_CUDA(cudaMemcpy(d_n, n_each, sizeof(int) * (size_t)B, cudaMemcpyHostToDevice));
+        ON_CUDA(cudaMemcpy(d_a, arrival, sizeof(int) * cells, cudaMemcpyHostToDevice));
+        ON_CUDA(cudaMemcpy(d_s, s, sizeof(int) * cells, cudaMemcpyHostToDevice));
+        ON_CUDA(cudaMemcpy(d_o, o, sizeof(int) * cells, cudaMemcpyHostToDevice));
+        ON_CUDA(cudaMemset(d_start, 0xff, sizeof(int) * cells));          // -1 where there is no request
+        ON_CUDA(cudaMemset(d_status, 0, sizeof(int)));
+        P.n_each = d_n; P.a = d_a; P.s = d_s; P.o = d_o; P.start_out = d_start; P.latency_out = d_lat; P.status = d_status;
+        ON_CUDA(cudaEventRecord(e0, 0));
+        k6_online<<<B, K6_THREADS, smem, 0>>>(P);
+        ON_CUDA(cudaGetLastError());
+        ON_CUDA(cudaEventRecord(e1, 0));
+        ON_CUDA(cudaDeviceSynchronize());
+        int status = 0;
+        ON_CUDA(cudaMemcpy(&status, d_status, sizeof(int), cudaMemcpyDeviceToHost));
+        if (status != 0) { rc = SCHED_E_INTERNAL; break; }
+        ON_CUDA(cudaMemcpy(start_out, d_start, sizeof(int) * cells, cudaMemcpyDeviceToHost));
+        ON_CUDA(cudaMemcpy(latency_out, d_lat, sizeof(i64) * (size_t)B, cudaMemcpyDeviceToHost));
+        if (kernel_ms_out) ON_CUDA(cudaEventElapsedTime(kernel_ms_out, e0, e1));
+#undef ON_CUDA
+    } while (0);
+    if (e0) cudaEventDestroy(e0);
+    if (e1) cudaEventDestroy(e1);
+    int* frees[] = {d_n, d_a, d_s, d_o, d_start, d_status};
+    for (int* ptr : frees) if (ptr) cudaFree(ptr);
+    if (d_lat) cudaFree(d_lat);
+    return rc;
 }
 
 int sched_stats(sched_handle h, int64_t* kernel_launches_out, int64_t* evaluations_out) {

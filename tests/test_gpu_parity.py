@@ -275,6 +275,91 @@ def test_sorted_f_quantile_greedy_matches_oracle():
         assert e.value.code == kv.E_UNSUPPORTED
 
 
+def _online_rows(instances):
+    n_max = max(len(x[0]) for x in instances)
+    B = len(instances)
+    a = np.zeros((B, n_max), dtype=np.int32); s = np.ones((B, n_max), dtype=np.int32); o = np.ones((B, n_max), dtype=np.int32)
+    n_each = np.zeros(B, dtype=np.int32)
+    for b, (ai, si, oi) in enumerate(instances):
+        n = len(ai)
+        n_each[b] = n
+        a[b, :n], s[b, :n], o[b, :n] = ai, si, oi
+    return n_each, a, s, o
+
+
+ONLINE = (kv.POLICY_FCFS, kv.POLICY_SOF, kv.POLICY_SORTED_F)
+
+
+def test_online_policies_match_oracle_on_small_streams():
+    """Section 6.2's online policies on many small arrival streams, several refresh periods and
+    look-ahead caps: every start time and every total latency."""
+    rng = np.random.default_rng(61)
+    M = 120
+    instances = []
+    for trial in range(48):
+        n = int(rng.integers(1, 70))
+        s, o = rand_instance(rng, n, M, M // 2, max(2, M // 4))
+        spread = int(rng.choice([0, n // 2 + 1, 3 * n, 20 * n]))           # all at once ... underloaded
+        a = np.sort(rng.integers(0, spread + 1, n)).astype(np.int32)
+        instances.append((a, s, o))
+    # the hand-worked streams of the CPU tests (M = 10 there; here they run in a launch of their own)
+    n_each, a, s, o = _online_rows(instances)
+    for policy in ONLINE:
+        for period, lookahead in ((10, 300), (1, 1), (3, 2), (7, 5), (1 << 30, 1000)):
+            starts, lat, _ = kv.online_simulate(n_each, a, s, o, M, policy, period, lookahead)
+            for b, (ai, si, oi) in enumerate(instances):
+                p, tot = orc.online_schedule(ai, si, oi, M, policy, period, lookahead)
+                n = len(ai)
+                assert (starts[b, :n] == p).all(), (policy, period, lookahead, b)
+                assert (starts[b, n:] == -1).all()
+                assert lat[b] == tot
+            if policy != kv.POLICY_SORTED_F:
+                break                                                     # the parameters only matter to Sorted-F-Online
+    hand = [([0, 0, 0, 1, 2, 6], [1, 1, 6, 1, 2, 3], [2, 2, 1, 1, 1, 2]), ([0, 0, 0, 0, 1], [5, 6, 6, 7, 1], [4, 3, 2, 2, 1])]
+    n_each, a, s, o = _online_rows(hand)
+    starts, lat, _ = kv.online_simulate(n_each, a, s, o, 10, kv.POLICY_SORTED_F, 3, 2)
+    assert starts[0].tolist() == [0, 0, 3, 2, 2, 6] and lat[0] == 13
+    starts, lat, _ = kv.online_simulate(n_each, a, s, o, 10, kv.POLICY_SORTED_F, 2, 10)
+    assert starts[1].tolist()[:5] == [7, 4, 0, 2, 2] and lat[1] == 26
+
+
+def test_online_poisson_streams_match_oracle():
+    """The paper's online experiment in small (Poisson arrivals, the three policies, period 10,
+    look-ahead 300) and two full-size streams (4000 iterations, rates 0.11 and 0.30)."""
+    streams = [W.online_poisson(lam, horizon=600, seed=20 + k) for k, lam in enumerate((0.05, 0.09, 0.13, 0.21, 0.30, 0.5))]
+    streams += [W.online_poisson(0.11, seed=31), W.online_poisson(0.30, seed=32)]
+    M = streams[0].M
+    n_each, a, s, o = _online_rows([(x.a, x.s, x.o) for x in streams])
+    totals = {}
+    for policy in ONLINE:
+        starts, lat, ms = kv.online_simulate(n_each, a, s, o, M, policy)
+        for b, x in enumerate(streams):
+            p, tot = orc.online_schedule(x.a, x.s, x.o, M, policy)
+            assert (starts[b, :x.n] == p).all(), (policy, x.name)
+            assert lat[b] == tot
+        totals[policy] = lat
+    # overloaded full-size stream: Sorted-F-Online < shortest decode first < FCFS (Section 7)
+    assert totals[kv.POLICY_SORTED_F][-1] < totals[kv.POLICY_SOF][-1] < totals[kv.POLICY_FCFS][-1]
+
+
+def test_online_argument_errors():
+    n_each, a, s, o = _online_rows([([0, 1], [2, 2], [1, 1])])
+    for bad in (dict(policy=kv.POLICY_TOTAL_SIZE), dict(period=0), dict(lookahead=0)):
+        args = dict(policy=kv.POLICY_FCFS, period=10, lookahead=300); args.update(bad)
+        with pytest.raises(kv.SchedError) as e:
+            kv.online_simulate(n_each, a, s, o, 10, args["policy"], args["period"], args["lookahead"])
+        assert e.value.code == kv.E_INVAL
+    with pytest.raises(kv.SchedError) as e:
+        kv.online_simulate(n_each, a[:, ::-1].copy(), s, o, 10, kv.POLICY_FCFS)        # arrivals decrease
+    assert e.value.code == kv.E_INVAL
+    with pytest.raises(kv.SchedError) as e:
+        kv.online_simulate(n_each, a, s, o, 2, kv.POLICY_FCFS)                          # s + o > M
+    assert e.value.code == kv.E_INVAL
+    with pytest.raises(kv.SchedError) as e:
+        kv.online_simulate(n_each, a, s, o, 10, kv.POLICY_SORTED_F, 10, 5000)           # look-ahead beyond the build's cap
+    assert e.value.code == kv.E_UNSUPPORTED
+
+
 def test_tiny_backlog_all_solvers_and_brute_force():
     """n = 16: prefix-F, Algorithm 4 and the exact DP orders, a full swap search from the DP order,
     and all 8! orders of the first 8 requests against the oracle's brute force."""
