@@ -295,3 +295,17 @@ def online_schedule(a, s, o, M, policy, period=10, lookahead=300):
     if rc != 0:
         raise ValueError("invalid online instance or parameters (%d)" % rc)
     return p, tot.value
+
+
+def amin_schedule(s, lower, o, M, order):
+    """Phase 2 of Sorted-F + A_min (Algorithm 6) on the given list with lower bounds ``lower`` of the
+    decode lengths.  Returns (final start times, TEL, evictions, peak memory actually used)."""
+    s, lower, o, order = _i32(s), _i32(lower), _i32(o), _i32(order)
+    n = len(s)
+    p = np.zeros(n, dtype=np.int64)
+    tel, ev, peak = C.c_longlong(0), C.c_longlong(0), C.c_longlong(0)
+    rc = lib().orc_amin_schedule(n, _p(s), _p(lower), _p(o), C.c_longlong(M), _p(order),
+                                 p.ctypes.data_as(C.c_void_p), C.byref(tel), C.byref(ev), C.byref(peak))
+    if rc != 0:
+        raise ValueError("invalid instance or iteration cap (%d)" % rc)
+    return p, tel.value, ev.value, peak.value

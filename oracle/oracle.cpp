@@ -5,7 +5,8 @@
 // Sorted-F (Section 3, Algorithm 1), the exact dynamic programme (Section 5.1, Algorithm 2),
 // Local Swap Search and Quantile Greedy Selection (Sections 5.2-5.3, Algorithms 4 and 5),
 // Sorted-G (Section 7), the online policies of Section 6.2 (FCFS, shortest decode first and
-// Sorted-F-Online under arrivals over time), and
+// Sorted-F-Online under arrivals over time), the executor of Sorted-F + A_min under lower-bound
+// predictions (Section 5.5, Algorithm 6), and
 // an order-level local search that scores every neighbour with Algorithm 1's Phase 2.  It exists
 // so that the GPU library can be checked against it; it shares no code with that library, is never
 // called by it, and nothing here is tuned for speed.  All arithmetic is integer.
@@ -842,6 +843,88 @@ int orc_online_schedule(int n, const int* a, const int* s, const int* o, i64 M, 
         for (int i = 0; i < n; ++i) tot += p_out[i] + o[i] - a[i];
         *total_latency = tot;
     }
+    return 0;
+}
+
+
+// ---------------------------------------------------------------------------------------------
+// O14. Sorted-F + A_min, Phase 2 (Section 5.5 "Handling Prediction Uncertainty", Algorithm 6):
+//      the executor when only a lower bound l_i <= o_i of every decode length is known.  Every
+//      request carries a running estimate e_i, initially l_i.  Iteration t = 1, 2, ...:
+//        1. requests that have run their o_i rounds leave; every other active request j is about
+//           to run its (t - p_j)-th round, so e_j <- max(e_j, t - p_j);
+//        2. admission as in Algorithm 1's Phase 2, on the estimates: the head r of the pending
+//           queue starts (p_r = t - 1) iff in every round tau >= t the PROJECTED memory
+//           sum over active j with p_j + e_j >= tau of (s_j + tau - p_j), r included, stays <= M;
+//           stop at the first head that does not fit;
+//        3. while the projected memory exceeds M in some round >= t, the active request with the
+//           smallest estimate (ties: lower index) is evicted: it loses its progress, keeps its
+//           estimate and goes back to the pending queue;
+//        4. the round runs.
+//      Left open by the listing and fixed here: the pending queue is always in the order of the
+//      given list (an evicted request returns to its place in that order, hence in front of
+//      everything not yet started); an evicted request restarts from scratch; estimates survive
+//      eviction.  The decisions never read o_i except to see that a request has finished.
+//      With l_i = o_i nothing is ever evicted and this is Algorithm 1's Phase 2.
+// Writes the final start times; tel = sum of (p_i + o_i); evictions = number of evictions;
+// peak = largest memory actually in use in any round (must be <= M).  Returns 0, or -2 if the
+// iteration cap is hit.
+// ---------------------------------------------------------------------------------------------
+int orc_amin_schedule(int n, const int* s, const int* lower, const int* o, i64 M, const int* order,
+                      i64* p_out, i64* tel_out, i64* evictions_out, i64* peak_out) {
+    if (n <= 0) return -1;
+    std::vector<int> pos(n, -1);
+    for (int q = 0; q < n; ++q) { if (order[q] < 0 || order[q] >= n || pos[order[q]] >= 0) return -1; pos[order[q]] = q; }
+    i64 cap = 16;
+    for (int i = 0; i < n; ++i) {
+        if (s[i] < 1 || o[i] < 1 || lower[i] < 1 || lower[i] > o[i] || (i64)s[i] + o[i] > M) return -1;
+        cap += (i64)o[i] * (n + 1);
+    }
+    std::vector<i64> est(lower, lower + n), p(n, -1);
+    std::vector<char> state(n, 0);                        // 0 pending, 1 active, 2 done
+    i64 evictions = 0, peak = 0;
+    int left = n;
+    auto projected_peak = [&](i64 t, int extra, i64 extra_p) {
+        i64 last = t;
+        for (int j = 0; j < n; ++j) if (state[j] == 1) last = std::max(last, p[j] + est[j]);
+        if (extra >= 0) last = std::max(last, extra_p + est[extra]);
+        i64 worst = 0;
+        for (i64 tau = t; tau <= last; ++tau) {
+            i64 u = 0;
+            for (int j = 0; j < n; ++j) if (state[j] == 1 && p[j] + est[j] >= tau) u += s[j] + tau - p[j];
+            if (extra >= 0 && extra_p + est[extra] >= tau) u += s[extra] + tau - extra_p;
+            worst = std::max(worst, u);
+        }
+        return worst;
+    };
+    for (i64 t = 1; left > 0; ++t) {
+        if (t > cap) return -2;
+        for (int j = 0; j < n; ++j) if (state[j] == 1) {
+            if (t - p[j] > o[j]) { state[j] = 2; --left; }
+            else est[j] = std::max(est[j], t - p[j]);
+        }
+        for (int q = 0; q < n; ++q) {                     // the pending queue, in list order
+            int r = order[q];
+            if (state[r] != 0) continue;
+            if (projected_peak(t, r, t - 1) > M) break;
+            state[r] = 1; p[r] = t - 1;
+        }
+        while (projected_peak(t, -1, 0) > M) {
+            int victim = -1;
+            for (int j = 0; j < n; ++j)
+                if (state[j] == 1 && (victim < 0 || est[j] < est[victim])) victim = j;
+            if (victim < 0) return -3;
+            state[victim] = 0; p[victim] = -1; ++evictions;
+        }
+        i64 used = 0;
+        for (int j = 0; j < n; ++j) if (state[j] == 1) used += s[j] + t - p[j];
+        peak = std::max(peak, used);
+    }
+    i64 tel = 0;
+    for (int i = 0; i < n; ++i) { p_out[i] = p[i]; tel += p[i] + o[i]; }
+    if (tel_out) *tel_out = tel;
+    if (evictions_out) *evictions_out = evictions;
+    if (peak_out) *peak_out = peak;
     return 0;
 }
 

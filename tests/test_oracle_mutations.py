@@ -53,6 +53,12 @@ MUTATIONS = [
     ("online: no look-ahead cap", "const int wn = m < lookahead ? m : lookahead;", "const int wn = m;", "test_sorted_f_online_worked_by_hand", False),
     ("online: periodic refresh never fires", "if (!computed || t - t_last >= period || was_empty", "if (!computed || was_empty",
      "test_sorted_f_online_worked_by_hand", False),
+    ("A_min evicts the largest estimate", "if (state[j] == 1 && (victim < 0 || est[j] < est[victim])) victim = j;",
+     "if (state[j] == 1 && (victim < 0 || est[j] > est[victim])) victim = j;", "test_amin_worked_by_hand", False),
+    ("A_min estimates never grow", "else est[j] = std::max(est[j], t - p[j]);", "else est[j] = est[j];",
+     "test_amin_never_exceeds_memory_and_finishes_everything", False),
+    ("A_min admission off by one", "if (projected_peak(t, r, t - 1) > M) break;", "if (projected_peak(t, r, t - 1) >= M) break;",
+     "test_amin_with_exact_predictions_is_algorithm_1", False),
     ("shortest-output-first sorts by size", "std::stable_sort(order, order + n, [&](int a, int b) { return o[a] < o[b]; });",
      "std::stable_sort(order, order + n, [&](int a, int b) { return s[a] + o[a] < s[b] + o[b]; });", "test_policies", False),
 ]

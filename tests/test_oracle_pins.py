@@ -756,3 +756,57 @@ def test_online_overload_ranking_of_the_three_policies():
     lat = {pol: orc.online_schedule(inst.a, inst.s, inst.o, inst.M, pol)[1] for pol in ONLINE_POLICIES}
     assert lat[orc.SORTED_F] < lat[orc.SOF] < lat[orc.FCFS]
     assert lat[orc.SORTED_F] < 0.5 * lat[orc.FCFS]
+
+
+# ---------------------------------------------------------------------------------------------
+# Sorted-F + A_min (Section 5.5, Algorithm 6): executor under lower-bound predictions
+# ---------------------------------------------------------------------------------------------
+def test_amin_with_exact_predictions_is_algorithm_1():
+    rng = np.random.default_rng(101)
+    for trial in range(15):
+        n = int(rng.integers(1, 40))
+        M = int(rng.integers(20, 200))
+        s, o = random_instance(rng, n, M, M // 2, max(2, M // 4))
+        order = rng.permutation(n).astype(np.int32)
+        p, tel, ev, peak = orc.amin_schedule(s, o, o, M, order)
+        rp, rtel, _ = orc.list_schedule_alg1(s, o, M, order)
+        assert (p == rp).all() and tel == rtel and ev == 0
+        assert peak == orc.check_schedule(s, o, M, rp)["peak"]
+
+
+def test_amin_never_exceeds_memory_and_finishes_everything():
+    rng = np.random.default_rng(102)
+    total_ev = 0
+    for trial in range(25):
+        n = int(rng.integers(2, 50))
+        M = int(rng.integers(30, 200))
+        s, o = random_instance(rng, n, M, M // 2, max(2, M // 3))
+        lower = np.maximum(1, np.floor(o * rng.uniform(0.1, 1.0, n))).astype(np.int32)
+        order = rng.permutation(n).astype(np.int32)
+        p, tel, ev, peak = orc.amin_schedule(s, lower, o, M, order)
+        total_ev += ev
+        assert peak <= M and (p >= 0).all() and tel == int((p + o).sum())
+        # the final runs alone (evicted attempts also used memory, so this is a lower bound on
+        # the peak) are a feasible schedule in the sense of the integer program
+        chk = orc.check_schedule(s, o, M, p)
+        assert chk["feasible"] and chk["peak"] <= peak
+    assert total_ev > 20                                # the eviction path really ran
+
+
+def test_amin_worked_by_hand():
+    # M = 8, list r0, r1.  r0 = (s 2, l 2, o 4), r1 = (s 3, l 1, o 2).
+    #  it 1: both start (projected round 1: 3 + 4).  it 2: both are in their 2nd round, estimates
+    #  2 and 2, round 2 would hold 4 + 5 = 9 > 8: equal estimates, the lower index r0 is evicted.
+    #  it 3: r1 has finished (c = 2); r0 starts again (p = 2) and runs 4 rounds: c = 6.
+    p, tel, ev, peak = orc.amin_schedule([2, 3], [2, 1], [4, 2], 8, [0, 1])
+    assert p.tolist() == [2, 0] and tel == 6 + 2 and ev == 1 and peak == 7
+    # r0 = (s 2, l 3, o 4), r1 = (s 3, l 1, o 3).
+    #  it 2: estimates 3 and 2, round 2 would hold 9: r1 (smaller estimate) is evicted, keeps 2.
+    #  it 3, 4: r1 refused (round 3: 5 + 4, round 4: 6 + 4).  it 5: r0 is done (c = 4), r1 starts
+    #  (p = 4), c = 7.
+    p, tel, ev, peak = orc.amin_schedule([2, 3], [3, 1], [4, 3], 8, [0, 1])
+    assert p.tolist() == [0, 4] and tel == 4 + 7 and ev == 1 and peak == 7
+    # an evicted request goes back IN FRONT of requests that never started: r2 = (s 1, l 1, o 1)
+    # is behind r1 in the list and must wait for it although it would fit in iteration 3
+    p, tel, ev, _ = orc.amin_schedule([2, 3, 1], [3, 1, 1], [4, 3, 1], 8, [0, 1, 2])
+    assert p.tolist() == [0, 4, 4] and ev == 1
