@@ -259,6 +259,44 @@ int sched_online_simulate(int32_t B, int32_t n_max, const int32_t* n_each, const
                           const int32_t* s, const int32_t* o, int64_t M, int32_t policy, int32_t period,
                           int32_t lookahead, int32_t* start_out, int64_t* latency_out, float* kernel_ms_out);
 
+/* Sorted-F + A_min, Phase 2 (Section 5.5, "Handling Prediction Uncertainty via Adaptive Output Length
+ * Refinement"; Algorithm 6 in Appendix D): B independent scenarios executed to completion when only a
+ * lower bound lower[i] <= o[i] of every decode length is known to the scheduler, one CTA per scenario.
+ * Scenario b has n_each[b] <= n_max requests in row b of the [B, n_max] arrays s / lower / o / order
+ * (entries past n_each[b] are ignored); order is the list to execute, a permutation of 0..n_each[b]-1
+ * (for the paper's method: Phase 1 run on the lower bounds).  Every request carries a running
+ * estimate, initially lower[i].  Iteration t = 1, 2, ...: (1) requests that have run o[i] rounds
+ * leave, every other running request's estimate becomes max(estimate, t - p_i); (2) pending requests
+ * are admitted in list order, p = t - 1, for as long as the memory projected from the estimates stays
+ * within M in every future round, stopping at the first that does not fit; (3) while the projection
+ * exceeds M the running request with the smallest estimate (ties: lower request index) is evicted --
+ * it loses its progress, keeps its estimate and returns to its place in the list; (4) the round runs.
+ * o[i] is used only to see that a request has finished.  With lower = o this is Algorithm 1's Phase 2.
+ *   start_out     : [B, n_max] final start time of every request, by request id (-1 where a row has
+ *                   no request).
+ *   tel_out       : [B] sum of (p_i + o_i).
+ *   evictions_out : [B] number of evictions, nullable.   peak_out : [B] largest memory actually in use
+ *                   in any round (never above M), nullable.   kernel_ms_out : device time, nullable.
+ * All pointers are host memory; the call allocates and frees its own device buffers and synchronises
+ * the device.  SCHED_E_INVAL: bad sizes, s < 1, lower < 1, lower > o, s + o > M;
+ * SCHED_E_NOT_PERMUTATION: a row of order is not a permutation; SCHED_E_UNSUPPORTED: n_max > 4096,
+ * o > 8192, M >= 2^30, or rows too large for the shared memory of one CTA (20 n_max + 16 L bytes,
+ * L = the power of two >= max o + 2); SCHED_E_INTERNAL: a scenario did not finish within
+ * 16 + (n+1) sum(o) rounds (capped at 2^30). */
+int sched_amin_simulate(int32_t B, int32_t n_max, const int32_t* n_each, const int32_t* s, const int32_t* lower,
+                        const int32_t* o, int64_t M, const int32_t* order, int32_t* start_out, int64_t* tel_out,
+                        int64_t* evictions_out, int64_t* peak_out, float* kernel_ms_out);
+
+/* Sorted-F + A_min end to end for one backlog (Algorithm 6): Phase 1 of Sorted-F on (s, lower) --
+ * phase1 = 0: prefix-F batch selection as in sched_sorted_f(); 1: Algorithm 4 as in
+ * sched_sorted_f_local_swap() -- then the executor of sched_amin_simulate() on the resulting list.
+ *   order_out : host int32[n], nullable, the Phase-1 list.  Other outputs as above with B = 1.
+ * Host pointers; creates and destroys a handle internally.  Errors as sched_init() and
+ * sched_amin_simulate(). */
+int sched_sorted_f_amin(int32_t n, const int32_t* s, const int32_t* lower, const int32_t* o, int64_t M,
+                        int32_t phase1, int32_t* order_out, int32_t* start_out, int64_t* tel_out,
+                        int64_t* evictions_out, int64_t* peak_out);
+
 /* Counters since sched_init: kernels launched by this handle, candidates evaluated. */
 int sched_stats(sched_handle h, int64_t* kernel_launches_out, int64_t* evaluations_out);
 

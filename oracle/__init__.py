@@ -309,3 +309,16 @@ def amin_schedule(s, lower, o, M, order):
     if rc != 0:
         raise ValueError("invalid instance or iteration cap (%d)" % rc)
     return p, tel.value, ev.value, peak.value
+
+
+def amin_schedule_rounds(s, lower, o, M, order):
+    """Same executor on a per-round array of projected memory (O14'); same return values."""
+    s, lower, o, order = _i32(s), _i32(lower), _i32(o), _i32(order)
+    n = len(s)
+    p = np.zeros(n, dtype=np.int64)
+    tel, ev, peak = C.c_longlong(0), C.c_longlong(0), C.c_longlong(0)
+    rc = lib().orc_amin_schedule_rounds(n, _p(s), _p(lower), _p(o), C.c_longlong(M), _p(order),
+                                        p.ctypes.data_as(C.c_void_p), C.byref(tel), C.byref(ev), C.byref(peak))
+    if rc != 0:
+        raise ValueError("invalid instance or iteration cap (%d)" % rc)
+    return p, tel.value, ev.value, peak.value

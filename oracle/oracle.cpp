@@ -22,7 +22,11 @@
 // "parity unpinned".  O12 (Algorithm 5): the routine is pinned for a GIVEN sample (hand-worked
 // cases, a library quantile, maximality), and the sampling hash to the generator's published
 // values; but which subset "random subset" means and how the 0.3-quantile of a finite sample is
-// read are choices no printed value fixes -- for those two choices: parity unpinned.
+// read are choices no printed value fixes -- for those two choices: parity unpinned.  O13 (online
+// arrivals) and O14 (Algorithm 6): the executors are pinned (reductions to the offline executor,
+// feasibility, hand-worked cases); which requests an online plan covers and where arrivals go, and
+// for Algorithm 6 where an evicted request re-enters the queue and how equal estimates are
+// ordered, are readings no printed value fixes -- for those choices: parity unpinned.
 #include <algorithm>
 #include <cstdint>
 #include <cstring>
@@ -919,6 +923,73 @@ int orc_amin_schedule(int n, const int* s, const int* lower, const int* o, i64 M
         i64 used = 0;
         for (int j = 0; j < n; ++j) if (state[j] == 1) used += s[j] + t - p[j];
         peak = std::max(peak, used);
+    }
+    i64 tel = 0;
+    for (int i = 0; i < n; ++i) { p_out[i] = p[i]; tel += p[i] + o[i]; }
+    if (tel_out) *tel_out = tel;
+    if (evictions_out) *evictions_out = evictions;
+    if (peak_out) *peak_out = peak;
+    return 0;
+}
+
+// ---------------------------------------------------------------------------------------------
+// O14'. The same executor on a per-round array of projected memory (proj[tau] = sum over running j
+//       with p_j + e_j >= tau of s_j + tau - p_j), so that instances of a few thousand requests
+//       can be checked: O14 re-derives every projection from the sets, which is cubic.  Same four
+//       steps in the same order; a grown estimate extends the projection by the current round, an
+//       admission adds the request's ramp over its estimated rounds, an eviction takes what is
+//       left of the victim's ramp away.  O14 is the definition; tests require O14' == O14 (start
+//       times, TEL, evictions, peak) on hundreds of instances before O14' is used for anything.
+// ---------------------------------------------------------------------------------------------
+int orc_amin_schedule_rounds(int n, const int* s, const int* lower, const int* o, i64 M, const int* order,
+                             i64* p_out, i64* tel_out, i64* evictions_out, i64* peak_out) {
+    if (n <= 0) return -1;
+    std::vector<int> pos(n, -1);
+    for (int q = 0; q < n; ++q) { if (order[q] < 0 || order[q] >= n || pos[order[q]] >= 0) return -1; pos[order[q]] = q; }
+    i64 cap = 16;
+    int omax = 1;
+    for (int i = 0; i < n; ++i) {
+        if (s[i] < 1 || o[i] < 1 || lower[i] < 1 || lower[i] > o[i] || (i64)s[i] + o[i] > M) return -1;
+        cap += (i64)o[i] * (n + 1);
+        omax = std::max(omax, o[i]);
+    }
+    const int H = omax + 2;                                // rounds t .. t+H-1 are kept, as a ring
+    std::vector<i64> proj(H, 0), est(lower, lower + n), p(n, -1);
+    std::vector<char> state(n, 0);
+    i64 evictions = 0, peak = 0;
+    int left = n;
+    for (i64 t = 1; left > 0; ++t) {
+        if (t > cap) return -2;
+        proj[(t - 1) % H] = 0;                             // round t-1 is over
+        for (int j = 0; j < n; ++j) if (state[j] == 1) {
+            if (t - p[j] > o[j]) { state[j] = 2; --left; }
+            else if (t - p[j] > est[j]) { est[j] = t - p[j]; proj[t % H] += s[j] + t - p[j]; }
+        }
+        for (int q = 0; q < n; ++q) {
+            const int r = order[q];
+            if (state[r] != 0) continue;
+            bool fits = true;
+            for (i64 tau = t; tau < t + H - 1 && fits; ++tau) {
+                i64 u = proj[tau % H];
+                if (tau <= t - 1 + est[r]) u += s[r] + tau - (t - 1);
+                if (u > M) fits = false;
+            }
+            if (!fits) break;
+            state[r] = 1; p[r] = t - 1;
+            for (i64 tau = t; tau <= t - 1 + est[r]; ++tau) proj[tau % H] += s[r] + tau - (t - 1);
+        }
+        for (;;) {
+            bool over = false;
+            for (i64 tau = t; tau < t + H - 1; ++tau) if (proj[tau % H] > M) over = true;
+            if (!over) break;
+            int victim = -1;
+            for (int k = 0; k < n; ++k)
+                if (state[k] == 1 && (victim < 0 || est[k] < est[victim])) victim = k;
+            if (victim < 0) return -3;
+            for (i64 tau = t; tau <= p[victim] + est[victim]; ++tau) proj[tau % H] -= s[victim] + tau - p[victim];
+            state[victim] = 0; p[victim] = -1; ++evictions;
+        }
+        peak = std::max(peak, proj[t % H]);
     }
     i64 tel = 0;
     for (int i = 0; i < n; ++i) { p_out[i] = p[i]; tel += p[i] + o[i]; }

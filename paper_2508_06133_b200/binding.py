@@ -22,7 +22,7 @@ NBHD_SWAP, NBHD_SWAP_INSERT, NBHD_SAMPLED = 0, 1, 2
 EXPORTS = [
     "sched_init", "sched_init_batch", "sched_set_stream", "sched_sync", "sched_set_prefill_weight", "sched_set_base_order",
     "sched_get_base_order", "sched_eval_batch", "sched_eval_batch_dev", "sched_sweep_dev",
-    "sched_sorted_f", "sched_sorted_f_dev", "sched_sorted_f_local_swap", "sched_sorted_f_local_swap_dev", "sched_sorted_f_dp", "sched_sorted_f_quantile", "sched_online_simulate", "sched_local_search", "sched_last_eval_kernel_ms", "sched_argmin_static_dev", "sched_stats", "sched_destroy",
+    "sched_sorted_f", "sched_sorted_f_dev", "sched_sorted_f_local_swap", "sched_sorted_f_local_swap_dev", "sched_sorted_f_dp", "sched_sorted_f_quantile", "sched_online_simulate", "sched_amin_simulate", "sched_sorted_f_amin", "sched_local_search", "sched_last_eval_kernel_ms", "sched_argmin_static_dev", "sched_stats", "sched_destroy",
     "sched_strerror", "sched_last_cuda_error",
 ]
 
@@ -69,6 +69,8 @@ def load():
     lib.sched_sorted_f_dp.argtypes = [vp, vp, vp, vp, vp]
     lib.sched_sorted_f_quantile.argtypes = [vp, C.c_uint64, vp, vp, vp, vp]
     lib.sched_online_simulate.argtypes = [i32, i32, vp, vp, vp, vp, i64, i32, i32, i32, vp, vp, vp]
+    lib.sched_amin_simulate.argtypes = [i32, i32, vp, vp, vp, vp, i64, vp, vp, vp, vp, vp, vp]
+    lib.sched_sorted_f_amin.argtypes = [i32, vp, vp, vp, i64, i32, vp, vp, vp, vp, vp]
     lib.sched_local_search.argtypes = [vp, C.c_int, i32, u64, i64, vp, vp, vp, vp]
     lib.sched_stats.argtypes = [vp, vp, vp]
     lib.sched_last_eval_kernel_ms.argtypes = [vp, vp]
@@ -301,3 +303,42 @@ def online_simulate(n_each, arrival, s, o, M, policy, period=10, lookahead=300):
                                         int(policy), int(period), int(lookahead), _np_ptr(starts), _np_ptr(lat), C.byref(ms)),
            "sched_online_simulate")
     return starts, lat, ms.value
+
+
+def amin_simulate(n_each, s, lower, o, M, order):
+    """B scenarios of Sorted-F + A_min's executor (rows of [B, n_max] arrays; see sched_amin_simulate).
+    Returns (start times [B, n_max], TEL [B], evictions [B], peak memory [B], kernel milliseconds)."""
+    s = np.ascontiguousarray(s, dtype=np.int32)
+    lower = np.ascontiguousarray(lower, dtype=np.int32)
+    o = np.ascontiguousarray(o, dtype=np.int32)
+    order = np.ascontiguousarray(order, dtype=np.int32)
+    n_each = np.ascontiguousarray(n_each, dtype=np.int32)
+    if s.ndim != 2 or lower.shape != s.shape or o.shape != s.shape or order.shape != s.shape or n_each.shape != (s.shape[0],):
+        raise ValueError("s, lower, o, order must be [B, n_max] and n_each [B]")
+    B, n_max = s.shape
+    starts = np.empty((B, n_max), dtype=np.int32)
+    tel = np.empty(B, dtype=np.int64)
+    ev = np.empty(B, dtype=np.int64)
+    peak = np.empty(B, dtype=np.int64)
+    ms = C.c_float(0.0)
+    _check(load().sched_amin_simulate(B, n_max, _np_ptr(n_each), _np_ptr(s), _np_ptr(lower), _np_ptr(o), int(M),
+                                      _np_ptr(order), _np_ptr(starts), _np_ptr(tel), _np_ptr(ev), _np_ptr(peak),
+                                      C.byref(ms)), "sched_amin_simulate")
+    return starts, tel, ev, peak, ms.value
+
+
+def sorted_f_amin(s, lower, o, M, phase1=0):
+    """Sorted-F + A_min for one backlog: Phase 1 on the lower bounds (0: prefix-F, 1: Algorithm 4), then
+    the adaptive executor.  Returns (order, start times, TEL, evictions, peak memory)."""
+    s = np.ascontiguousarray(s, dtype=np.int32)
+    lower = np.ascontiguousarray(lower, dtype=np.int32)
+    o = np.ascontiguousarray(o, dtype=np.int32)
+    if s.ndim != 1 or lower.shape != s.shape or o.shape != s.shape:
+        raise ValueError("s, lower, o must be 1-D arrays of one length")
+    n = s.shape[0]
+    order = np.empty(n, dtype=np.int32)
+    starts = np.empty(n, dtype=np.int32)
+    tel, ev, peak = C.c_int64(0), C.c_int64(0), C.c_int64(0)
+    _check(load().sched_sorted_f_amin(n, _np_ptr(s), _np_ptr(lower), _np_ptr(o), int(M), int(phase1), _np_ptr(order),
+                                      _np_ptr(starts), C.byref(tel), C.byref(ev), C.byref(peak)), "sched_sorted_f_amin")
+    return order, starts, tel.value, ev.value, peak.value

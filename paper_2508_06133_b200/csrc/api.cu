@@ -17,6 +17,7 @@
 #include "k3_eval.cuh"
 #include "k5_argmin.cuh"
 #include "k6_online.cuh"
+#include "k7_amin.cuh"
 
 thread_local char g_last_cuda_error[256] = "";
 
@@ -955,6 +956,129 @@ int sched_online_simulate(int32_t B, int32_t n_max, const int32_t* n_each, const
     int* frees[] = {d_n, d_a, d_s, d_o, d_start, d_status};
     for (int* ptr : frees) if (ptr) cudaFree(ptr);
     if (d_lat) cudaFree(d_lat);
+    return rc;
+}
+
+// Shared by the two A_min entry points: validates the scenarios on the host, stages them, runs k7_amin.
+// order_host: [B, n_max] host lists, or NULL when order_dev (one device row of n_max entries) is given.
+static int amin_run(int32_t B, int32_t n_max, const int32_t* n_each, const int32_t* s, const int32_t* lower,
+                    const int32_t* o, int64_t M, const int32_t* order_host, const int32_t* order_dev,
+                    int32_t* start_out, int64_t* tel_out, int64_t* evictions_out, int64_t* peak_out,
+                    float* kernel_ms_out) {
+    if (B < 1 || n_max < 1 || !n_each || !s || !lower || !o || (!order_host && !order_dev) || !start_out || !tel_out)
+        return SCHED_E_INVAL;
+    if (M < 2) return SCHED_E_INVAL;
+    if (n_max > K7_MAX_N || M >= (1ll << 30)) return SCHED_E_UNSUPPORTED;
+    int omax = 1;
+    std::vector<unsigned char> seen;
+    for (int b = 0; b < B; ++b) {
+        const int n = n_each[b];
+        if (n < 1 || n > n_max) return SCHED_E_INVAL;
+        const size_t base = (size_t)b * n_max;
+        for (int i = 0; i < n; ++i) {
+            const int si = s[base + i], oi = o[base + i], li = lower[base + i];
+            if (si < 1 || oi < 1 || li < 1 || li > oi || (i64)si + oi > M) return SCHED_E_INVAL;
+            omax = oi > omax ? oi : omax;
+        }
+        if (order_host) {
+            seen.assign((size_t)n, 0);
+            for (int q = 0; q < n; ++q) {
+                const int id = order_host[base + q];
+                if (id < 0 || id >= n || seen[id]) return SCHED_E_NOT_PERMUTATION;
+                seen[id] = 1;
+            }
+        }
+    }
+    if (omax > K7_MAX_O) return SCHED_E_UNSUPPORTED;
+    AminParams P;
+    memset(&P, 0, sizeof(P));
+    P.n_max = n_max; P.M = (int)M;
+    P.L = 32; while (P.L < omax + 2) P.L <<= 1;
+    const size_t smem = sizeof(int) * ((size_t)5 * n_max + (size_t)4 * P.L);
+    int dev = 0, optin = 0;
+    KV_CUDA(cudaGetDevice(&dev));
+    KV_CUDA(cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+    if (smem + 1024 > (size_t)optin) return SCHED_E_UNSUPPORTED;
+    KV_CUDA(cudaFuncSetAttribute(k7_amin, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+
+    const size_t cells = (size_t)B * n_max;
+    int *d_n = nullptr, *d_s = nullptr, *d_l = nullptr, *d_o = nullptr, *d_ord = nullptr, *d_start = nullptr, *d_status = nullptr;
+    i64* d_res = nullptr;                                   // tel | evictions | peak, B each
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    int rc = SCHED_OK;
+    do {
+#define AM_CUDA(call) if ((call) != cudaSuccess) { rc = kv_cuda_fail(cudaGetLastError(), #call); break; }
+        if ((rc = dev_alloc(&d_n, (size_t)B)) != SCHED_OK) break;
+        if ((rc = dev_alloc(&d_s, cells)) != SCHED_OK) break;
+        if ((rc = dev_alloc(&d_l, cells)) != SCHED_OK) break;
+        if ((rc = dev_alloc(&d_o, cells)) != SCHED_OK) break;
+        if (order_host && (rc = dev_alloc(&d_ord, cells)) != SCHED_OK) break;
+        if ((rc = dev_alloc(&d_start, cells)) != SCHED_OK) break;
+        if ((rc = dev_alloc(&d_res, (size_t)3 * B)) != SCHED_OK) break;
+        if ((rc = dev_alloc(&d_status, 1)) != SCHED_OK) break;
+        AM_CUDA(cudaEventCreate(&e0));
+        AM_CUDA(cudaEventCreate(&e1));
+        AM_CUDA(cudaMemcpy(d_n, n_each, sizeof(int) * (size_t)B, cudaMemcpyHostToDevice));
+        AM_CUDA(cudaMemcpy(d_s, s, sizeof(int) * cells, cudaMemcpyHostToDevice));
+        AM_CUDA(cudaMemcpy(d_l, lower, sizeof(int) * cells, cudaMemcpyHostToDevice));
+        AM_CUDA(cudaMemcpy(d_o, o, sizeof(int) * cells, cudaMemcpyHostToDevice));
+        if (order_host) AM_CUDA(cudaMemcpy(d_ord, order_host, sizeof(int) * cells, cudaMemcpyHostToDevice));
+        AM_CUDA(cudaMemset(d_start, 0xff, sizeof(int) * cells));           // -1 where a row has no request
+        AM_CUDA(cudaMemset(d_status, 0, sizeof(int)));
+        P.n_each = d_n; P.s = d_s; P.lower = d_l; P.o = d_o;
+        P.order = order_host ? d_ord : order_dev;
+        P.order_stride = order_host ? (size_t)n_max : 0;
+        P.start_out = d_start; P.tel_out = d_res; P.evict_out = d_res + B; P.peak_out = d_res + 2 * (size_t)B;
+        P.status = d_status;
+        AM_CUDA(cudaEventRecord(e0, 0));
+        k7_amin<<<B, K7_THREADS, smem, 0>>>(P);
+        AM_CUDA(cudaGetLastError());
+        AM_CUDA(cudaEventRecord(e1, 0));
+        AM_CUDA(cudaDeviceSynchronize());
+        int status = 0;
+        AM_CUDA(cudaMemcpy(&status, d_status, sizeof(int), cudaMemcpyDeviceToHost));
+        if (status != 0) { rc = SCHED_E_INTERNAL; break; }
+        AM_CUDA(cudaMemcpy(start_out, d_start, sizeof(int) * cells, cudaMemcpyDeviceToHost));
+        AM_CUDA(cudaMemcpy(tel_out, d_res, sizeof(i64) * (size_t)B, cudaMemcpyDeviceToHost));
+        if (evictions_out) AM_CUDA(cudaMemcpy(evictions_out, d_res + B, sizeof(i64) * (size_t)B, cudaMemcpyDeviceToHost));
+        if (peak_out) AM_CUDA(cudaMemcpy(peak_out, d_res + 2 * (size_t)B, sizeof(i64) * (size_t)B, cudaMemcpyDeviceToHost));
+        if (kernel_ms_out) AM_CUDA(cudaEventElapsedTime(kernel_ms_out, e0, e1));
+#undef AM_CUDA
+    } while (0);
+    if (e0) cudaEventDestroy(e0);
+    if (e1) cudaEventDestroy(e1);
+    int* frees[] = {d_n, d_s, d_l, d_o, d_ord, d_start, d_status};
+    for (int* ptr : frees) if (ptr) cudaFree(ptr);
+    if (d_res) cudaFree(d_res);
+    return rc;
+}
+
+int sched_amin_simulate(int32_t B, int32_t n_max, const int32_t* n_each, const int32_t* s, const int32_t* lower,
+                        const int32_t* o, int64_t M, const int32_t* order, int32_t* start_out, int64_t* tel_out,
+                        int64_t* evictions_out, int64_t* peak_out, float* kernel_ms_out) {
+    if (!order) return SCHED_E_INVAL;
+    return amin_run(B, n_max, n_each, s, lower, o, M, order, nullptr, start_out, tel_out, evictions_out, peak_out,
+                    kernel_ms_out);
+}
+
+int sched_sorted_f_amin(int32_t n, const int32_t* s, const int32_t* lower, const int32_t* o, int64_t M,
+                        int32_t phase1, int32_t* order_out, int32_t* start_out, int64_t* tel_out,
+                        int64_t* evictions_out, int64_t* peak_out) {
+    if (n < 1 || !s || !lower || !o || !start_out || !tel_out) return SCHED_E_INVAL;
+    if (phase1 != 0 && phase1 != 1) return SCHED_E_INVAL;
+    for (int i = 0; i < n; ++i)
+        if (s[i] < 1 || o[i] < 1 || lower[i] < 1 || lower[i] > o[i] || (i64)s[i] + o[i] > M) return SCHED_E_INVAL;
+    // Phase 1 sees the lower bounds in place of the decode lengths
+    sched_handle h = nullptr;
+    KV_TRY(sched_init(&h, n, s, lower, M));
+    int rc = sorted_f_common_dev(h, phase1, nullptr, nullptr, nullptr, nullptr);
+    if (rc == SCHED_OK) rc = sched_sync(h);
+    if (rc == SCHED_OK && order_out &&
+        cudaMemcpy(order_out, h->d_order, sizeof(int) * (size_t)n, cudaMemcpyDeviceToHost) != cudaSuccess)
+        rc = kv_cuda_fail(cudaGetLastError(), "cudaMemcpy(order_out)");
+    if (rc == SCHED_OK)
+        rc = amin_run(1, n, &n, s, lower, o, M, nullptr, h->d_order, start_out, tel_out, evictions_out, peak_out, nullptr);
+    sched_destroy(h);
     return rc;
 }
 

@@ -360,6 +360,101 @@ def test_online_argument_errors():
     assert e.value.code == kv.E_UNSUPPORTED
 
 
+def _amin_rows(instances):
+    """instances: list of (s, lower, o, order) -> padded [B, n_max] rows."""
+    n_max = max(len(x[0]) for x in instances)
+    B = len(instances)
+    s = np.ones((B, n_max), dtype=np.int32); lo = np.ones((B, n_max), dtype=np.int32); o = np.ones((B, n_max), dtype=np.int32)
+    order = np.zeros((B, n_max), dtype=np.int32)
+    n_each = np.zeros(B, dtype=np.int32)
+    for b, (si, li, oi, ordi) in enumerate(instances):
+        n = len(si)
+        n_each[b] = n
+        s[b, :n], lo[b, :n], o[b, :n], order[b, :n] = si, li, oi, ordi
+    return n_each, s, lo, o, order
+
+
+def test_amin_small_scenarios_match_the_set_form_oracle():
+    """Algorithm 6's executor against the oracle that re-derives every projection from the sets:
+    every final start time, TEL, eviction count and peak memory; tight and loose memories, exact,
+    mild and crude lower bounds (l = 1 for everybody included), and the hand-worked cases."""
+    rng = np.random.default_rng(71)
+    for M in (60, 150):
+        instances = []
+        for trial in range(60):
+            n = int(rng.integers(1, 60))
+            s, o = rand_instance(rng, n, M, M // 2, max(2, M // int(rng.integers(2, 6))))
+            kind = trial % 4
+            if kind == 0: lower = o.copy()
+            elif kind == 1: lower = np.ones(n, dtype=np.int32)
+            else: lower = np.clip(np.floor(o * rng.uniform(0.0 if kind == 2 else 0.6, 1.0, n)), 1, o).astype(np.int32)
+            instances.append((s, lower, o, rng.permutation(n).astype(np.int32)))
+        n_each, s, lo, o, order = _amin_rows(instances)
+        starts, tel, ev, peak, _ = kv.amin_simulate(n_each, s, lo, o, M, order)
+        total_ev = 0
+        for b, (si, li, oi, ordi) in enumerate(instances):
+            p, rtel, rev, rpeak = orc.amin_schedule(si, li, oi, M, ordi)
+            n = len(si)
+            assert (starts[b, :n] == p).all(), (M, b)
+            assert (starts[b, n:] == -1).all()
+            assert (tel[b], ev[b], peak[b]) == (rtel, rev, rpeak), (M, b)
+            if b % 4 == 0:
+                assert ev[b] == 0
+            total_ev += rev
+        assert total_ev > 100
+    hand = [([2, 3], [2, 1], [4, 2], [0, 1]), ([2, 3], [3, 1], [4, 3], [0, 1]), ([2, 3, 1], [3, 1, 1], [4, 3, 1], [0, 1, 2])]
+    n_each, s, lo, o, order = _amin_rows(hand)
+    starts, tel, ev, peak, _ = kv.amin_simulate(n_each, s, lo, o, 8, order)
+    assert starts[0, :2].tolist() == [2, 0] and (tel[0], ev[0], peak[0]) == (8, 1, 7)
+    assert starts[1, :2].tolist() == [0, 4] and (tel[1], ev[1], peak[1]) == (11, 1, 7)
+    assert starts[2].tolist() == [0, 4, 4] and ev[2] == 1
+
+
+def test_amin_backlogs_of_paper_size_match_the_per_round_oracle():
+    """Backlogs of the size of the paper's experiments (n = 2000, M = 16,492) and of the 1,000-request
+    mixture, lists from Phase 1 on the lower bounds, interval predictions of several widths
+    (l = ceil(gamma o)): the whole of Sorted-F + A_min against the oracle (Phase 1 on the lower
+    bounds, then the per-round executor); with exact predictions it is Sorted-F itself."""
+    for inst, gammas in ((W.paper_scale(), (1.0, 0.8, 0.5)), (W.mixed_1k(), (0.9, 0.3))):
+        rng = np.random.default_rng(5)
+        for gamma in gammas:
+            lower = np.clip(np.ceil(inst.o * rng.uniform(gamma, 1.0, inst.n)), 1, inst.o).astype(np.int32)
+            for phase1 in (0, 1):
+                order, starts, tel, ev, peak = kv.sorted_f_amin(inst.s, lower, inst.o, inst.M, phase1)
+                if phase1 == 0:
+                    r_order = orc.sorted_f_prefix(inst.s, lower, inst.M)[0]
+                else:
+                    r_order = orc.sorted_f_local_swap(inst.s, lower, inst.M)[0]
+                assert (order == r_order).all()
+                p, rtel, rev, rpeak = orc.amin_schedule_rounds(inst.s, lower, inst.o, inst.M, r_order)
+                assert (starts == p).all() and (tel, ev, peak) == (rtel, rev, rpeak), (inst.name, gamma, phase1)
+                assert peak <= inst.M
+                if gamma == 1.0:
+                    assert ev == 0 and tel == orc.list_schedule_rounds(inst.s, inst.o, inst.M, r_order)[1]
+                else:
+                    assert ev > 0
+
+
+def test_amin_argument_errors():
+    n_each, s, lo, o, order = _amin_rows([([2, 3], [1, 1], [4, 2], [0, 1])])
+    with pytest.raises(kv.SchedError) as e:
+        kv.amin_simulate(n_each, s, o + 1, o, 8, order)                     # lower bound above the length
+    assert e.value.code == kv.E_INVAL
+    with pytest.raises(kv.SchedError) as e:
+        kv.amin_simulate(n_each, s, lo, o, 5, order)                        # s + o > M
+    assert e.value.code == kv.E_INVAL
+    with pytest.raises(kv.SchedError) as e:
+        kv.amin_simulate(n_each, s, lo, o, 8, np.zeros_like(order))         # not a permutation
+    assert e.value.code == kv.E_NOT_PERMUTATION
+    big = np.full((1, 2), 9000, dtype=np.int32)
+    with pytest.raises(kv.SchedError) as e:
+        kv.amin_simulate(n_each, s, big, big, 1 << 20, order)               # decode beyond the build's cap
+    assert e.value.code == kv.E_UNSUPPORTED
+    with pytest.raises(kv.SchedError) as e:
+        kv.sorted_f_amin([2, 3], [1, 1], [4, 2], 8, phase1=7)
+    assert e.value.code == kv.E_INVAL
+
+
 def test_tiny_backlog_all_solvers_and_brute_force():
     """n = 16: prefix-F, Algorithm 4 and the exact DP orders, a full swap search from the DP order,
     and all 8! orders of the first 8 requests against the oracle's brute force."""

@@ -59,6 +59,12 @@ MUTATIONS = [
      "test_amin_never_exceeds_memory_and_finishes_everything", False),
     ("A_min admission off by one", "if (projected_peak(t, r, t - 1) > M) break;", "if (projected_peak(t, r, t - 1) >= M) break;",
      "test_amin_with_exact_predictions_is_algorithm_1", False),
+    ("per-round A_min leaves an evicted ramp behind", "for (i64 tau = t; tau <= p[victim] + est[victim]; ++tau) proj[tau % H] -= s[victim] + tau - p[victim];",
+     "for (i64 tau = t + 1; tau <= p[victim] + est[victim]; ++tau) proj[tau % H] -= s[victim] + tau - p[victim];",
+     "test_amin_per_round_form_equals_the_set_form", False),
+    ("per-round A_min grows an estimate without its memory", "else if (t - p[j] > est[j]) { est[j] = t - p[j]; proj[t % H] += s[j] + t - p[j]; }",
+     "else if (t - p[j] > est[j]) { est[j] = t - p[j]; proj[t % H] += t - p[j]; }",
+     "test_amin_per_round_form_equals_the_set_form", False),
     ("shortest-output-first sorts by size", "std::stable_sort(order, order + n, [&](int a, int b) { return o[a] < o[b]; });",
      "std::stable_sort(order, order + n, [&](int a, int b) { return s[a] + o[a] < s[b] + o[b]; });", "test_policies", False),
 ]

@@ -810,3 +810,25 @@ def test_amin_worked_by_hand():
     # is behind r1 in the list and must wait for it although it would fit in iteration 3
     p, tel, ev, _ = orc.amin_schedule([2, 3, 1], [3, 1, 1], [4, 3, 1], 8, [0, 1, 2])
     assert p.tolist() == [0, 4, 4] and ev == 1
+
+
+def test_amin_per_round_form_equals_the_set_form():
+    """O14' (projected memory kept per round) against O14 (projection re-derived from the sets):
+    start times, TEL, evictions and peak, over tight and loose memories and crude lower bounds."""
+    rng = np.random.default_rng(103)
+    evs = 0
+    for trial in range(300):
+        n = int(rng.integers(1, 45))
+        M = int(rng.integers(12, 160))
+        s, o = random_instance(rng, n, M, max(1, M // 2), max(2, M // int(rng.integers(2, 6))))
+        frac = rng.uniform(0.0, 1.0) if trial % 3 else 0.0
+        lower = np.clip(np.floor(o * rng.uniform(frac, 1.0, n)), 1, o).astype(np.int32)
+        order = rng.permutation(n).astype(np.int32)
+        a = orc.amin_schedule(s, lower, o, M, order)
+        b = orc.amin_schedule_rounds(s, lower, o, M, order)
+        assert (a[0] == b[0]).all() and a[1:] == b[1:], trial
+        evs += a[2]
+    assert evs > 300
+    # the worked cases
+    assert orc.amin_schedule_rounds([2, 3], [2, 1], [4, 2], 8, [0, 1])[0].tolist() == [2, 0]
+    assert orc.amin_schedule_rounds([2, 3, 1], [3, 1, 1], [4, 3, 1], 8, [0, 1, 2])[0].tolist() == [0, 4, 4]
