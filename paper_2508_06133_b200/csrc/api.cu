@@ -32,9 +32,12 @@ const i64 kSweepChunk = 1ll << 22;          // candidates per launch inside a sw
 const size_t kSnapBudget = 512ull << 20;    // bytes of snapshot memory before striding kicks in
 
 // Runs CALL(SIM) with SIM = the simulator class of the handle: the register-resident one when the
-// longest window fits 33 registers per lane, else the shared-memory one.
+// longest window fits 33 registers per lane, else the hybrid one (registers + a shared-memory ring
+// for the far rounds); the all-shared-memory one on request (KVSCHED_SIM=smem).
 #define KV_DISPATCH_SIM(h, CALL)                               \
-    if ((h)->nreg > 0) {                                        \
+    if ((h)->hyb) {                                             \
+        CALL(HybSim);                                           \
+    } else if ((h)->nreg > 0) {                                      \
         switch ((h)->nreg) {                                    \
             case 2: CALL(RegSim<2>); break;                     \
             case 3: CALL(RegSim<3>); break;                     \
@@ -136,15 +139,15 @@ int k3_warps(const sched_ctx* h) {
 #define GETW(SIM) w = SIM::kWarps
     KV_DISPATCH_SIM(h, GETW);
 #undef GETW
-    if (h->nreg == 0) {                       // one ring per warp has to fit in shared memory
-        const int fit = (int)(((size_t)h->smem_optin - 2048) / ((size_t)h->L * sizeof(int)));
+    if (h->ring_cells > 0) {                  // one ring per warp has to fit in shared memory
+        const int fit = (int)(((size_t)h->smem_optin - 2048) / ((size_t)h->ring_cells * sizeof(int)));
         if (fit < w) w = fit;
     }
     return w;
 }
 
 size_t k3_smem_bytes(const sched_ctx* h, bool* table_in_smem, unsigned* table_bytes) {
-    const size_t rings = h->nreg > 0 ? 0 : (size_t)k3_warps(h) * h->L * sizeof(int);
+    const size_t rings = (size_t)k3_warps(h) * h->ring_cells * sizeof(int);
     const unsigned tb = (unsigned)(((size_t)h->n * sizeof(int2) + 15) & ~(size_t)15);
     const size_t with_table = ((size_t)tb + 127) / 128 * 128 + rings;
     if (with_table <= (size_t)h->smem_optin - 2048) {
@@ -181,8 +184,11 @@ int create_common(sched_ctx** out, int B, int n, const int32_t* s, const int32_t
         h->B = B; h->n = n; h->M = M; h->omax = omax; h->sum_o_max = sum_max;
         h->g_num = 0; h->g_den = 1;
         h->nreg = sim_pick_nreg(omax);
-        if (const char* kind = getenv("KVSCHED_SIM"))               // testing knob: "smem" forces the shared-memory simulator
-            if (strcmp(kind, "smem") == 0) h->nreg = 0;
+        h->hyb = h->nreg == 0;
+        if (const char* kind = getenv("KVSCHED_SIM")) {             // testing knob: "smem" / "hybrid" force that simulator
+            if (strcmp(kind, "smem") == 0) { h->nreg = 0; h->hyb = false; }
+            if (strcmp(kind, "hybrid") == 0) { h->nreg = 0; h->hyb = true; }
+        }
         h->nit = sim_pick_nit(omax);
         if (const char* cap = getenv("KVSCHED_MAX_NIT")) {          // tuning knob: windows beyond the cap stream
             const int c = atoi(cap);
@@ -190,7 +196,8 @@ int create_common(sched_ctx** out, int B, int n, const int32_t* s, const int32_t
         }
         // cells per simulator state: registers x 32 lanes, or a ring whose length is a multiple of
         // 32 cells (a wrapped 16-byte access then keeps its bank)
-        h->L = h->nreg > 0 ? 32 * h->nreg : (omax + 8 + 31) & ~31;
+        h->L = h->hyb ? 32 * (HybSim::NREG + sim_pick_far_chunks(omax)) : h->nreg > 0 ? 32 * h->nreg : (omax + 8 + 31) & ~31;
+        h->ring_cells = h->hyb ? HybSim::ring_cells(h->L) : h->nreg > 0 ? 0 : h->L;
         if (k3_warps(h) < 1) { rc = SCHED_E_UNSUPPORTED; break; }
         if (cudaStreamCreateWithFlags(&h->own_stream, cudaStreamNonBlocking) != cudaSuccess) { rc = kv_cuda_fail(cudaGetLastError(), "cudaStreamCreate"); break; }
         h->stream = h->own_stream;
@@ -267,7 +274,7 @@ int ensure_base(sched_ctx* h) {
     const int n = h->n;
     k3_gather_table<<<(n + 255) / 256, 256, 0, h->stream>>>(h->d_tbl_id, h->d_order, n, h->d_tbl_base);
     KV_TRY(check_launch(h));
-#define RUN(N) k3_base_run<N><<<1, 32, (size_t)h->L * sizeof(int), h->stream>>>(                   \
+#define RUN(N) k3_base_run<N><<<1, 32, (size_t)h->ring_cells * sizeof(int), h->stream>>>(                  \
         h->d_tbl_base, n, h->L, (int)h->M, h->snap_stride, h->d_snap_ring, h->d_snap_hdr,            \
         h->d_base_starts, h->d_base_tel, h->d_status)
     KV_DISPATCH_SIM(h, RUN);
@@ -434,7 +441,7 @@ int sched_eval_batch_dev(sched_handle h, int kind, int64_t count, const void* ca
     const int n = h->n;
     if (kind == SCHED_CAND_POLICY) {
         const size_t smem = (size_t)(n + 1) * 16 + (size_t)n * 8 + (size_t)n * 16 + (size_t)(n + 2) * 4 +
-                            (h->nreg > 0 ? 0 : (size_t)h->L * 4);
+                            (size_t)h->ring_cells * 4;
         if (smem > (size_t)h->smem_optin - 2048) return SCHED_E_UNSUPPORTED;
         const i64 ctas = (i64)h->B * count;
         if (ctas >= (1ll << 31)) return SCHED_E_UNSUPPORTED;

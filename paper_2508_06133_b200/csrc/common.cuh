@@ -28,9 +28,11 @@ struct sched_ctx {
     int B, n;                // instances, requests per instance
     i64 M;
     int omax;                // largest decode length over all instances
-    int L;                   // cells per simulator state (32 * nreg, or a ring of a multiple of 32 cells >= omax + 8)
+    int L;                   // cells per simulator state (32 * nreg; 32 * (33 + far chunks); or a ring of a multiple of 32 cells >= omax + 8)
     int nreg;                // > 0: register-resident simulator with this many registers per lane
     int nit;                 // shared-memory simulator: 128-cell rounds cached in registers (0: streamed)
+    bool hyb;                // hybrid simulator: 33 registers per lane + a shared-memory ring for the rounds after them
+    int ring_cells;          // shared-memory ints one simulator needs (0 for the register simulator)
     i64 sum_o_max;           // largest sum of o over instances (bounds every start time)
     int sm_count;
     int smem_optin;          // max dynamic shared memory per block (bytes)

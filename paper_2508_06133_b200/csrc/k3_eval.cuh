@@ -22,6 +22,7 @@
 #include "k4_moves.cuh"
 #include "sim.cuh"
 #include "sim_reg.cuh"
+#include "sim_hyb.cuh"
 
 #define K3S_WARPS 16                       // warps per CTA of the start-time checker
 
@@ -94,7 +95,7 @@ __global__ void k3_iota(int* a, int n) {
 
 // ------------------------------------------------------------------------------------------------
 // Base run: positions 0 .. n-1 of the base order; snapshot idx holds the state in front of
-// position idx * stride.  One warp.  Dynamic shared memory: L ints (shared-memory simulator only).
+// position idx * stride.  One warp.  Dynamic shared memory: the simulator's ring, if it has one.
 // ------------------------------------------------------------------------------------------------
 template <class SIM>
 __global__ void __launch_bounds__(32)
@@ -166,7 +167,7 @@ k3_eval_moves(const MoveEvalParams p) {
     if (slot >= p.count) return;
     const i64 c = p.launch_order[slot];
     SIM sim;
-    sim.attach((int*)(smem_raw + ring_off) + (size_t)warp * L, L);
+    sim.attach((int*)(smem_raw + ring_off) + (size_t)warp * SIM::ring_cells(L), L);
     const Move mv = k4_move_of(p.src, n, c);
     if ((unsigned)mv.i >= (unsigned)n || (unsigned)mv.j >= (unsigned)n) {      // code outside the neighbourhood
         if (lane == 0) p.tel_out[c] = INT64_MAX;
@@ -232,7 +233,7 @@ k3_eval_orders(const OrderEvalParams p) {
     const i64 c = (i64)blockIdx.x * (blockDim.x >> 5) + warp;      // every order has the same length
     if (c >= p.count) return;
     SIM sim;
-    sim.attach((int*)(smem_raw + ring_off) + (size_t)warp * L, L);
+    sim.attach((int*)(smem_raw + ring_off) + (size_t)warp * SIM::ring_cells(L), L);
     const int* ord = p.orders + (size_t)c * n;
     int* starts = kStarts ? p.starts_out + (size_t)c * n : nullptr;
     sim.reset(lane);
@@ -258,7 +259,7 @@ k3_eval_orders(const OrderEvalParams p) {
 
 // ------------------------------------------------------------------------------------------------
 // Policy sweep: grid = B * P single-warp CTAs; CTA (b, k) evaluates instance b under policies[k].
-// Dynamic shared memory: int ring[L] (shared-memory simulator only; L = 0 otherwise); i64 P[n+1],
+// Dynamic shared memory: the simulator's ring (SIM::ring_cells(L) ints); i64 P[n+1],
 // O[n+1]; u64 key[n]; int s[n], o[n], ord[n], tmp[n], boff[n+2].
 // ------------------------------------------------------------------------------------------------
 __device__ __forceinline__ void k3_rank_sort(const u64* key, const int* ids_in, int* ids_out, int lo, int hi, int lane) {
@@ -285,7 +286,7 @@ k3_eval_policy(const int* __restrict__ s_all, const int* __restrict__ o_all, int
     const int b = blockIdx.x / num_policies, kpol = blockIdx.x % num_policies;
     const int policy = policies[kpol];
     int* ring = (int*)smem_raw;                       // first: 16-byte aligned for the vector loads
-    i64* P = (i64*)(ring + (SIM::kUsesSmem ? L : 0)); // L is a multiple of 4
+    i64* P = (i64*)(ring + SIM::ring_cells(L));       // a multiple of 4
     i64* O = P + (n + 1);
     u64* key = (u64*)(O + (n + 1));
     int* s = (int*)(key + n);

@@ -218,6 +218,7 @@ __device__ __forceinline__ int sim_admit(int* __restrict__ ring, int L, int M, S
 template <int NIT>
 struct SmemSim {
     static constexpr bool kUsesSmem = true;
+    __host__ __device__ static constexpr int ring_cells(int L) { return L; }   // shared-memory ints per warp
     static constexpr int kWarps = 24;                 // warps per CTA of the persistent kernels
     int* ring;
     int L;

@@ -57,6 +57,7 @@ struct RegSim {
     static_assert(NREG >= 2 && NREG <= 33, "the bucket tree covers up to 33 registers");
     static constexpr int kCells = 32 * NREG;
     static constexpr bool kUsesSmem = false;
+    __host__ __device__ static constexpr int ring_cells(int) { return 0; }   // shared-memory ints per warp
     // warps per CTA of the persistent kernels, limited by the register file (64K / threads)
 #ifndef KV_REG33_WARPS
 #define KV_REG33_WARPS 32

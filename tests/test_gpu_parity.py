@@ -80,7 +80,7 @@ def test_orders_long_waits_and_ring_wrap():
 
 @pytest.mark.parametrize("omax", [100, 127, 128, 129, 255, 256, 257, 511, 512, 513, 1023, 1024, 1025, 1500, 3000])
 def test_orders_every_simulator_shape(omax):
-    """Window lengths around each register-cached shape's limit, and the streamed shape beyond."""
+    """Window lengths around each register count's limit, and the hybrid simulator beyond 1025."""
     rng = np.random.default_rng(omax)
     n, M = 90, 4 * omax
     s = rng.integers(1, omax, n).astype(np.int32)
@@ -97,6 +97,45 @@ def test_orders_every_simulator_shape(omax):
         p, tt, _ = orc.list_schedule_rounds(s, o, M, orders[c])
         assert tel[c] == tt and (starts[c] == p).all()
     assert (mtel == oracle_moves(s, o, M, orders[0], codes)).all()
+
+
+@pytest.mark.parametrize("sim", ["smem", "hybrid"])
+def test_simulators_with_shared_memory_timelines(sim, monkeypatch):
+    """The all-shared-memory simulator and the hybrid one (33 registers per lane + a shared-memory ring
+    for the rounds after them), each forced for every window length: short windows that never reach
+    the ring, windows that end in its first chunk, windows over most of it, waits longer than the
+    whole state; explicit orders with start times, moves from snapshots, and the policy sweep."""
+    monkeypatch.setenv("KVSCHED_SIM", sim)
+    for omax in (1, 3, 40, 300, 1025, 1026, 1057, 1100, 2500, 4096):
+        rng = np.random.default_rng(1000 + omax)
+        n, M = 70, 4 * omax + 8
+        s = rng.integers(1, M - omax, n).astype(np.int32)
+        o = rng.integers(1, omax + 1, n).astype(np.int32)
+        o[:6] = [omax, max(1, omax - 1), 1, min(2, omax), min(33, omax), omax]
+        s[::9] = M - o[::9]                                   # requests that need the machine alone
+        orders = np.stack([rng.permutation(n) for _ in range(3)]).astype(np.int32)
+        with kv.Scheduler(s, o, M) as h:
+            tel, _, starts = h.eval_batch(kv.CAND_ORDER, orders, want_starts=True)
+            h.set_base_order(orders[0])
+            codes = all_codes(n)[::53]
+            mtel, _, _ = h.eval_batch(kv.CAND_MOVE, codes)
+        for c in range(3):
+            p, tt, _ = orc.list_schedule_rounds(s, o, M, orders[c])
+            assert tel[c] == tt and (starts[c] == p).all(), (sim, omax, c)
+        assert (mtel == oracle_moves(s, o, M, orders[0], codes)).all(), (sim, omax)
+    # policy sweep (one single-warp CTA per instance and policy) on the same simulator class
+    rng = np.random.default_rng(77)
+    B, n, M = 6, 60, 6000
+    s = rng.integers(1, 3000, (B, n)).astype(np.int32)
+    o = rng.integers(1, 1500, (B, n)).astype(np.int32)
+    pol = np.array([kv.POLICY_FCFS, kv.POLICY_SOF, kv.POLICY_TOTAL_SIZE, kv.POLICY_SORTED_F], dtype=np.int32)
+    with kv.Scheduler.batch(s, o, M) as h:
+        tel, _, _ = h.eval_batch(kv.CAND_POLICY, pol)
+    for b in range(B):
+        refs = [orc.policy_order(s[b], o[b], orc.FCFS), orc.policy_order(s[b], o[b], orc.SHORTEST_OUTPUT_FIRST),
+                orc.policy_order(s[b], o[b], orc.TOTAL_SIZE_FIRST), orc.sorted_f_prefix(s[b], o[b], M)[0]]
+        for k, order in enumerate(refs):
+            assert tel[b, k] == orc.list_schedule_rounds(s[b], o[b], M, order)[1], (sim, b, k)
 
 
 def test_orders_mixed_1k():
@@ -713,7 +752,7 @@ def test_mixed_1k_swap_search_to_local_optimum():
 
 
 def test_heavy_100k_backlog():
-    """n = 100,000, o up to 4,096 (shared-memory simulator, strided snapshots), int64 TELs."""
+    """n = 100,000, o up to 4,096 (hybrid simulator, strided snapshots), int64 TELs."""
     inst = W.heavy_100k()
     n = inst.n
     with kv.Scheduler(inst.s, inst.o, inst.M) as h:
