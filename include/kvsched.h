@@ -207,6 +207,23 @@ int sched_local_search(sched_handle h, int neighbourhood, int32_t iters, uint64_
                        int64_t samples_per_iter, int32_t* order_inout, int64_t* tel_out,
                        int32_t* iters_done_out, int64_t* trace_out);
 
+/* One acceptance step of the order-level local search for callers that run the neighbourhood sweep
+ * themselves, e.g. split over several GPUs: every GPU sweeps its share of the move indices with
+ * sched_sweep_dev(), the (TEL, index) pairs are reduced to the smallest one (ties: lower index) and
+ * every GPU then makes this call with the same pair, so that all base orders stay identical.
+ * The move is accepted iff best_tel is strictly below the TEL of the current base order (Section 5.2's
+ * improving rule); it is then applied to the base order on the device and the base run with its
+ * snapshots is rebuilt.
+ *   best_tel, best_index : the winning pair; best_index is a move code (sampled = 0, SWAP_INSERT
+ *                          coding) or the sample number m of iteration `iteration` under `seed`.
+ *   accepted_out         : 1 if the move was applied, else 0; nullable.
+ *   tel_out              : TEL of the base order after the call; nullable.
+ * Synchronises the handle's stream.  SCHED_E_INVAL: batch handle, n < 2, index outside the
+ * neighbourhood.  SCHED_E_INTERNAL: the applied move does not reproduce best_tel (the pair did not
+ * come from a sweep of this base order). */
+int sched_accept_move(sched_handle h, int64_t best_tel, int64_t best_index, int sampled, uint64_t seed,
+                      int32_t iteration, int32_t* accepted_out, int64_t* tel_out);
+
 /* Device time, in milliseconds, of the most recent schedule-simulation kernel launch of this handle
  * (the move / order evaluator), measured with CUDA events recorded on the handle's stream around
  * that launch.  Waits for the launch to finish.  SCHED_E_INVAL if there was none. */

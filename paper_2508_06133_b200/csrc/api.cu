@@ -877,6 +877,38 @@ int sched_local_search(sched_handle h, int neighbourhood, int32_t iters, uint64_
     return read_status(h);
 }
 
+int sched_accept_move(sched_handle h, int64_t best_tel, int64_t best_index, int sampled, uint64_t seed,
+                      int32_t iteration, int32_t* accepted_out, int64_t* tel_out) {
+    KV_ENTER(h);
+    if (h->batch_handle || h->n < 2 || best_index < 0 || iteration < 0) return SCHED_E_INVAL;
+    const int n = h->n;
+    if (!sampled && best_index >= neighbourhood_size(n, SCHED_NBHD_SWAP_INSERT, 0)) return SCHED_E_INVAL;
+    cudaStream_t st = h->stream;
+    KV_TRY(ensure_base(h));
+    i64* d_cur = (i64*)h->d_state;               // {current TEL, accepted flag}
+    int* d_acc = (int*)(d_cur + 1);
+    i64* hp = (i64*)h->h_pinned;                 // {best TEL, best index, accepted, base TEL}
+    hp[0] = best_tel; hp[1] = best_index;
+    KV_CUDA(cudaMemcpyAsync(h->d_best, hp, 2 * sizeof(i64), cudaMemcpyHostToDevice, st));
+    KV_CUDA(cudaMemcpyAsync(d_cur, h->d_base_tel, sizeof(i64), cudaMemcpyDeviceToDevice, st));
+    k5_accept_move<<<1, 256, 0, st>>>(h->d_order, n, h->d_best, d_cur, d_acc, h->d_vals_b, sampled ? 1 : 0, seed, iteration);
+    KV_TRY(check_launch(h));
+    KV_CUDA(cudaMemcpyAsync(&hp[2], d_acc, sizeof(int), cudaMemcpyDeviceToHost, st));
+    KV_CUDA(cudaStreamSynchronize(st));
+    const bool accepted = *(int*)&hp[2] != 0;
+    if (accepted) {
+        h->base_ready = false;
+        KV_TRY(ensure_base(h));
+    }
+    KV_CUDA(cudaMemcpyAsync(&hp[3], h->d_base_tel, sizeof(i64), cudaMemcpyDeviceToHost, st));
+    KV_CUDA(cudaStreamSynchronize(st));
+    // the re-simulated order must reproduce the TEL that the caller's sweep reported for this move
+    if (accepted && hp[3] != best_tel) return SCHED_E_INTERNAL;
+    if (accepted_out) *accepted_out = accepted ? 1 : 0;
+    if (tel_out) *tel_out = hp[3];
+    return read_status(h);
+}
+
 int sched_last_eval_kernel_ms(sched_handle h, float* ms_out) {
     KV_ENTER(h);
     if (!ms_out || !h->ev_valid) return SCHED_E_INVAL;

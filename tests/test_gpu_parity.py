@@ -651,6 +651,44 @@ def test_local_search_first_sweeps_mixed_1k():
     assert oracle_moves(inst.s, inst.o, inst.M, base, codes).min() >= trace[0][1]
 
 
+def test_sharded_search_driver_on_one_gpu_equals_the_library_search():
+    """parallel.sharded_local_search with one rank (sweep + sched_accept_move per iteration) against
+    sched_local_search and the oracle; then the same search with the sweep cut into three shares that
+    are reduced on the host, which is what several ranks do."""
+    from paper_2508_06133_b200 import parallel as par
+    rng = np.random.default_rng(91)
+    n, M = 40, 300
+    s, o = rand_instance(rng, n, M, 120, 60)
+    start = rng.permutation(n).astype(np.int32)
+    for nbhd, iters, samples in ((kv.NBHD_SWAP_INSERT, 60, 0), (kv.NBHD_SAMPLED, 12, 200)):
+        r_order, r_tel, r_done, r_trace = orc.local_search(s, o, M, nbhd, iters, start, seed=3, samples=samples)
+        with kv.Scheduler(s, o, M) as h:
+            h.set_base_order(start)
+            tel, done, trace = par.sharded_local_search(par.GpuEvaluator(h), nbhd, iters, seed=3, samples_per_iter=samples)
+            assert (tel, done) == (r_tel, r_done) and (trace == r_trace).all()
+            assert (h.get_base_order() == r_order).all()
+        with kv.Scheduler(s, o, M) as h:                       # three shares, reduced as the ranks would
+            h.set_base_order(start)
+            ev = par.GpuEvaluator(h)
+            total = par.neighbourhood_size(n, nbhd, samples)
+            for it in range(r_done):
+                pairs = [ev.sweep(*par.shard(total, r, 3), nbhd == kv.NBHD_SAMPLED, 3, it) for r in range(3)]
+                best = min(pairs)                              # smallest TEL, then lowest index
+                assert (best[1], best[0]) == tuple(r_trace[it])
+                ev.accept(best[0], best[1], nbhd == kv.NBHD_SAMPLED, 3, it)
+            assert (h.get_base_order() == r_order).all()
+    with kv.Scheduler(s, o, M) as h:
+        h.set_base_order(start)
+        base = orc.list_schedule_rounds(s, o, M, start)[1]
+        assert h.accept_move(base, 0) == (False, base)         # not strictly better: refused
+        with pytest.raises(kv.SchedError) as e:
+            h.accept_move(base - 1, 0)                         # a TEL that move 0 does not have
+        assert e.value.code == kv.E_INTERNAL
+        with pytest.raises(kv.SchedError) as e:
+            h.accept_move(1, n * (n - 1) // 2 + n * (n - 1))   # index outside the neighbourhood
+        assert e.value.code == kv.E_INVAL
+
+
 def test_device_pointer_candidates_are_bounds_checked_on_the_device():
     import torch
     dev = torch.device("cuda", torch.cuda.current_device())
