@@ -28,8 +28,9 @@
 //   break it, and only in round t: "the projection exceeds M" is occ[t] > M.
 //   While the head of the queue is refused nothing is admitted and occ only grows, so the bound on
 //   its wait that the window test gives (a cell over budget by x at offset r needs min(x, r+1) more
-//   rounds) stays valid until the next eviction.  Rounds in which nothing can happen (no overflow,
-//   head still bound to wait) are walked by one thread, a handful of instructions each.
+//   rounds) stays valid until the next eviction.  Rounds in which nothing can happen (no overflow;
+//   head still bound to wait, or not even its first round fits) are walked by one thread, a handful
+//   of instructions each.
 #pragma once
 
 #include "common.cuh"
@@ -160,6 +161,7 @@ __global__ void __launch_bounds__(K7_THREADS) k7_amin(const AminParams P) {
         if (tid == 0) {
             // rounds in which nothing can be decided: step 1 only
             int act = K7_ACT_WORK;
+            const int head_s = head < n ? ps[head] : 0;
             for (;;) {
                 const int k = t & mask;
                 cnt += (unsigned)dc[k]; A += dA[k]; remaining -= fin[k];
@@ -167,7 +169,9 @@ __global__ void __launch_bounds__(K7_THREADS) k7_amin(const AminParams P) {
                 const int u = occ[k] + (int)(A + cnt * (unsigned)t);
                 occ[k] = u;
                 if (remaining == 0) { act = K7_ACT_DONE; break; }
-                if (u > M || (head < n && t >= t_ok)) break;
+                // the head's first round is the current one: if it does not fit there, the window
+                // test cannot succeed in this iteration and the CTA need not be woken for it
+                if (u > M || (head < n && t >= t_ok && u + head_s + 1 <= M)) break;
                 if ((i64)t >= round_cap) { act = K7_ACT_CAP; break; }
                 peak = max(peak, u);
                 occ[k] = 0;
