@@ -38,7 +38,7 @@ FALLBACK_HBM_GBS, FALLBACK_SM_MHZ = 6650.0, 1965.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one simulator launch, from a one-pass ncu capture of
 # this very launch (profiles/k3_eval_moves_mixed_n10000_dram_traffic.md); keyed by (workload, moves per
 # launch, simulator source files' digest) so that it turns into null when the kernel changes
-K3_TRAFFIC = {("mixed_n10000", 1 << 18): (43.28e6 + 512.0, "cb282219dec17532")}
+K3_TRAFFIC = {("mixed_n10000", 1 << 22): (60.61e6 + 11.38e6, "21db94945fc6e5e0")}
 
 
 def simulator_digest() -> str:
@@ -180,7 +180,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--moves", type=int, default=1 << 18, help="sampled moves evaluated per step and GPU")
+    ap.add_argument("--moves", type=int, default=1 << 22, help="sampled moves evaluated per step and GPU")
     ap.add_argument("--ref-moves", type=int, default=96, help="moves per step of the CPU reference arm")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="mixed_10k", choices=["mixed_10k", "mixed_1k", "paper_scale"])
@@ -271,7 +271,7 @@ def main():
     roof_alu = {"bound": "alu", "achieved": alu_ach, "peak": alu_peak, "unit": "Tint-op/s", "frac": alu_ach / alu_peak}
     roofline = dict(roof_alu)
     ring_cells = (int(inst.o.max()) + 8 + 31) & ~31
-    hbm_bytes = 4.0 * n * ring_cells + 8.0 * count + 8.0 * n      # snapshots read once, TELs out, request table
+    hbm_bytes = 4.0 * n * ring_cells + 8.0 * count + 4.0 * count + 8.0 * n   # snapshots read once, TELs out, launch order in, request table
     traffic = None
     known = K3_TRAFFIC.get((inst.name, count))
     if known is not None and known[1] == simulator_digest():

@@ -313,8 +313,10 @@ int order_candidates(sched_ctx* h, const MoveSource& src, i64 count) {
     return SCHED_OK;
 }
 
+// by_slot: TELs are left in launch-slot order (h->d_k4's launch_order maps a slot to its candidate
+// until the next call); the sweeps that only need the arg-min use it, see launch_argmin.
 int launch_moves(sched_ctx* h, int mode, const i64* codes, i64 first, u64 seed, int iteration,
-                 i64 count, i64* tel_out, int* starts_out) {
+                 i64 count, i64* tel_out, int* starts_out, bool by_slot = false) {
     if (count <= 0) return SCHED_OK;
     if (count >= (1ll << 31)) return SCHED_E_UNSUPPORTED;
     KV_TRY(ensure_base(h));
@@ -326,7 +328,7 @@ int launch_moves(sched_ctx* h, int mode, const i64* codes, i64 first, u64 seed, 
     p.tbl_base = h->d_tbl_base; p.table_in_smem = in_smem ? 1 : 0; p.table_bytes = tb;
     p.snap_ring = h->d_snap_ring; p.snap_hdr = h->d_snap_hdr;
     p.src.mode = mode; p.src.codes = codes; p.src.first = first; p.src.seed = seed; p.src.iteration = iteration;
-    p.count = count; p.tel_out = tel_out; p.starts_out = starts_out;
+    p.count = count; p.tel_out = tel_out; p.tel_by_slot = by_slot ? 1 : 0; p.starts_out = starts_out;
     p.base_order = h->d_order; p.base_starts_pos = h->d_base_starts;
     p.status = h->d_status;
     KV_TRY(order_candidates(h, p.src, count));
@@ -344,12 +346,15 @@ int launch_moves(sched_ctx* h, int mode, const i64* codes, i64 first, u64 seed, 
     return SCHED_OK;
 }
 
-int launch_argmin(sched_ctx* h, const i64* tel, i64 count, i64 index_base, const i64* prior, i64* best_out) {
+const int* last_launch_order(const sched_ctx* h, i64 count) { return (const int*)h->d_k4 + h->n + 1 + count; }
+
+int launch_argmin(sched_ctx* h, const i64* tel, i64 count, i64 index_base, const i64* prior, i64* best_out,
+                  const int* index_map = nullptr) {
     i64 blocks = (count / 2 + K5_THREADS - 1) / K5_THREADS;
     if (blocks < 1) blocks = 1;
     if (blocks > 4 * h->sm_count) blocks = 4 * h->sm_count;
     if (blocks > 4096) blocks = 4096;
-    k5_argmin<<<(unsigned)blocks, K5_THREADS, 0, h->stream>>>(tel, count, index_base, prior, h->d_partials, h->d_ticket, best_out);
+    k5_argmin<<<(unsigned)blocks, K5_THREADS, 0, h->stream>>>(tel, count, index_base, index_map, prior, h->d_partials, h->d_ticket, best_out);
     return check_launch(h);
 }
 
@@ -587,8 +592,10 @@ int sched_sweep_dev(sched_handle h, int sampled, uint64_t seed, int32_t iteratio
         i64* dst;
         if (tel) dst = tel + done;
         else { KV_TRY(ensure_tel(h, c)); dst = h->d_tel; }
-        KV_TRY(launch_moves(h, sampled ? 2 : 1, nullptr, first_code + done, seed, iteration, c, dst, nullptr));
-        KV_TRY(launch_argmin(h, dst, c, first_code + done, done ? (const i64*)best_out : nullptr, (i64*)best_out));
+        const bool by_slot = tel == nullptr;       // nobody reads the scratch TELs by candidate index
+        KV_TRY(launch_moves(h, sampled ? 2 : 1, nullptr, first_code + done, seed, iteration, c, dst, nullptr, by_slot));
+        KV_TRY(launch_argmin(h, dst, c, first_code + done, done ? (const i64*)best_out : nullptr, (i64*)best_out,
+                             by_slot ? last_launch_order(h, c) : nullptr));
     }
     return SCHED_OK;
 }
@@ -848,8 +855,8 @@ int sched_local_search(sched_handle h, int neighbourhood, int32_t iters, uint64_
         KV_TRY(ensure_tel(h, total < kSweepChunk ? total : kSweepChunk));
         for (i64 done = 0; done < total; done += kSweepChunk) {
             const i64 c = total - done < kSweepChunk ? total - done : kSweepChunk;
-            KV_TRY(launch_moves(h, sampled ? 2 : 1, nullptr, done, seed, it, c, h->d_tel, nullptr));
-            KV_TRY(launch_argmin(h, h->d_tel, c, done, done ? h->d_best : nullptr, h->d_best));
+            KV_TRY(launch_moves(h, sampled ? 2 : 1, nullptr, done, seed, it, c, h->d_tel, nullptr, true));
+            KV_TRY(launch_argmin(h, h->d_tel, c, done, done ? h->d_best : nullptr, h->d_best, last_launch_order(h, c)));
         }
         k5_accept_move<<<1, 256, 0, st>>>(h->d_order, n, h->d_best, d_cur, d_acc, h->d_vals_b, sampled, seed, it);
         KV_TRY(check_launch(h));

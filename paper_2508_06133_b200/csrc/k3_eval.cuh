@@ -139,6 +139,8 @@ struct MoveEvalParams {
     i64 count;
     const int* launch_order;           // candidate index of every launch slot (K4)
     i64* tel_out;
+    int tel_by_slot;                   // 1: tel_out is indexed by launch slot (full-sector writes; the arg-min maps
+                                       // slots back through launch_order), 0: by candidate index
     int* starts_out;                   // nullable [count][n], by request id
     const int* base_order;
     const int* base_starts_pos;
@@ -166,11 +168,12 @@ k3_eval_moves(const MoveEvalParams p) {
     const i64 slot = (i64)blockIdx.x * (blockDim.x >> 5) + warp;
     if (slot >= p.count) return;
     const i64 c = p.launch_order[slot];
+    i64* tel_dst = p.tel_out + (p.tel_by_slot ? slot : c);
     SIM sim;
     sim.attach((int*)(smem_raw + ring_off) + (size_t)warp * SIM::ring_cells(L), L);
     const Move mv = k4_move_of(p.src, n, c);
     if ((unsigned)mv.i >= (unsigned)n || (unsigned)mv.j >= (unsigned)n) {      // code outside the neighbourhood
-        if (lane == 0) p.tel_out[c] = INT64_MAX;
+        if (lane == 0) *tel_dst = INT64_MAX;
         return;
     }
     const int first_pos = min(mv.i, mv.j);
@@ -197,7 +200,7 @@ k3_eval_moves(const MoveEvalParams p) {
             if (kStarts && lane == k) starts[id] = pstart;
         }
     }
-    if (lane == 0) p.tel_out[c] = sim.total();
+    if (lane == 0) *tel_dst = sim.total();
 }
 
 // ------------------------------------------------------------------------------------------------

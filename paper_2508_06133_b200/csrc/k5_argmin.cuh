@@ -5,7 +5,8 @@
 // values, the smallest index -- the pair never depends on the order in which threads arrive.
 // TELs are read as 16-byte vectors, reduced per warp with shuffles, per block through shared
 // memory, and the last block to finish (ticket counter) folds the per-block partials and an
-// optional earlier result (`prior`, for sweeps evaluated in several launches).
+// optional earlier result (`prior`, for sweeps evaluated in several launches).  With `index_map` the
+// array is in launch-slot order and element k belongs to index index_base + index_map[k].
 #pragma once
 
 #include "common.cuh"
@@ -17,7 +18,7 @@ __device__ __forceinline__ void k5_take(i64& bv, i64& bi, i64 v, i64 i) {
 }
 
 __global__ void __launch_bounds__(K5_THREADS)
-k5_argmin(const i64* __restrict__ tel, i64 count, i64 index_base, const i64* prior,
+k5_argmin(const i64* __restrict__ tel, i64 count, i64 index_base, const int* __restrict__ index_map, const i64* prior,
           i64* __restrict__ partials, unsigned int* ticket, i64* __restrict__ best_out) {
     __shared__ i64 sh_v[K5_THREADS / 32], sh_i[K5_THREADS / 32];
     __shared__ bool is_last;
@@ -27,10 +28,11 @@ k5_argmin(const i64* __restrict__ tel, i64 count, i64 index_base, const i64* pri
     const longlong2* tel2 = reinterpret_cast<const longlong2*>(tel);      // cudaMalloc'd: 16-byte aligned
     for (i64 k = (i64)blockIdx.x * K5_THREADS + tid; k < pairs; k += (i64)gridDim.x * K5_THREADS) {
         const longlong2 v = tel2[k];
-        k5_take(bv, bi, v.x, index_base + 2 * k);
-        k5_take(bv, bi, v.y, index_base + 2 * k + 1);
+        k5_take(bv, bi, v.x, index_base + (index_map ? (i64)index_map[2 * k] : 2 * k));
+        k5_take(bv, bi, v.y, index_base + (index_map ? (i64)index_map[2 * k + 1] : 2 * k + 1));
     }
-    if ((count & 1) && blockIdx.x == 0 && tid == 0) k5_take(bv, bi, tel[count - 1], index_base + count - 1);
+    if ((count & 1) && blockIdx.x == 0 && tid == 0)
+        k5_take(bv, bi, tel[count - 1], index_base + (index_map ? (i64)index_map[count - 1] : count - 1));
     for (int d = 16; d >= 1; d >>= 1) {
         const i64 ov = __shfl_xor_sync(KV_FULL, bv, d), oi = __shfl_xor_sync(KV_FULL, bi, d);
         k5_take(bv, bi, ov, oi);

@@ -195,19 +195,23 @@ def test_moves_sampled_codes_mixed_1k_and_10k():
 
 
 def test_sweep_in_the_benchmarks_launch_configuration():
-    """The launch the benchmark times: one sweep of 262,144 sampled moves of the Sorted-F order of the
-    10,000-request backlog on the handle's stream.  Sampled outputs against the oracle one by one;
-    the reduced (TEL, index) pair against an arg-min of the dumped TELs on the host; and, as a
-    property that holds at any size, no candidate beats the sum of decode lengths."""
+    """The launch the benchmark times: one sweep of 4,194,304 sampled moves of the Sorted-F order of
+    the 10,000-request backlog on the handle's stream, reduced to its best (TEL, index) pair without
+    a per-candidate output (TELs stay in launch-slot order inside the library).  The same sweep
+    with the TELs dumped: sampled outputs against the oracle one by one; the reduced pair of both
+    sweeps against an arg-min of the dumped TELs on the host; and, as a property that holds at
+    any size, no candidate beats the sum of decode lengths."""
     import torch
     inst = W.mixed_10k()
-    count, seed, it = 1 << 18, 20250806, 3
+    count, seed, it = 1 << 22, 20250806, 3
     dev = torch.device("cuda", 0)
     tel = torch.empty(count, dtype=torch.int64, device=dev)
     best = torch.zeros(2, dtype=torch.int64, device=dev)
+    best_dump = torch.zeros(2, dtype=torch.int64, device=dev)
     with kv.Scheduler(inst.s, inst.o, inst.M) as h:
         h.sorted_f_dev()
-        h.sweep_dev(count, best, sampled=True, seed=seed, iteration=it, first_code=0, tel_out=tel)
+        h.sweep_dev(count, best, sampled=True, seed=seed, iteration=it, first_code=0)
+        h.sweep_dev(count, best_dump, sampled=True, seed=seed, iteration=it, first_code=0, tel_out=tel)
         h.sync()
         order = h.get_base_order()
     tels = tel.cpu().numpy()
@@ -218,6 +222,7 @@ def test_sweep_in_the_benchmarks_launch_configuration():
     ref = orc.eval_moves(inst.s, inst.o, inst.M, r_order, [m[0] for m in mv], [m[1] for m in mv], [m[2] for m in mv])
     assert (tels[picks] == ref).all()
     k = int(np.argmin(tels))                                   # first minimum = lowest index
+    assert best_dump.cpu().tolist() == [int(tels[k]), k]
     assert best.cpu().tolist() == [int(tels[k]), k]
     assert tels.min() >= int(inst.o.sum())                     # every request completes no earlier than its own o
 
