@@ -12,8 +12,8 @@ def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run on the B200 box)")
 
 
-@pytest.fixture(scope="session")
-def golden():
+def load_golden():
+    """Values the paper prints (tests/golden/paper_values.txt: name | value | where it is printed)."""
     vals = {}
     with open(os.path.join(ROOT, "tests", "golden", "paper_values.txt")) as f:
         for line in f:
@@ -23,3 +23,8 @@ def golden():
             name, value, _where = [x.strip() for x in line.split("|", 2)]
             vals[name] = int(value)
     return vals
+
+
+@pytest.fixture(scope="session")
+def golden():
+    return load_golden()

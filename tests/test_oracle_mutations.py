@@ -4,6 +4,7 @@ fails.  A pin that still passed would mean that part of the oracle is effectivel
 import ctypes as C
 import os
 import subprocess
+import sys
 
 import pytest
 
@@ -75,27 +76,46 @@ def source():
     return open(SRC).read()
 
 
+_CHILD = r"""
+import ctypes as C, sys
+sys.path.insert(0, sys.argv[1])
+import oracle as orc
+from tests import test_oracle_pins as pins
+from tests.conftest import load_golden
+lib = C.CDLL(sys.argv[2])
+lib.orc_bruteforce_opt.restype = C.c_longlong
+lib.orc_bruteforce_best_order.restype = C.c_longlong
+orc.lib()                      # the real library first, so that nothing rebuilds it later
+orc._lib = lib
+pin, needs_golden = sys.argv[3], sys.argv[4] == "1"
+gold = load_golden() if needs_golden else None
+fn = getattr(pins, pin)
+try:
+    if pin == "test_example1_tel":
+        for ex in (orc.list_schedule_alg1, orc.list_schedule_rounds):
+            fn(gold, ex)
+    elif needs_golden:
+        fn(gold)
+    else:
+        fn()
+except (AssertionError, ValueError):
+    sys.exit(0)                # the pin caught the planted mistake
+sys.exit(3)                    # the pin still passes
+"""
+
+
 @pytest.mark.parametrize("what,old,new,pin,needs_golden", MUTATIONS, ids=[m[0] for m in MUTATIONS])
-def test_pin_catches_planted_mistake(tmp_path, source, golden, what, old, new, pin, needs_golden):
+def test_pin_catches_planted_mistake(tmp_path, source, what, old, new, pin, needs_golden):
+    """The mutated copy runs in a child process: a planted mistake may write out of bounds, and a
+    fault there must not take the test session down.  Exit code 0 = the pin failed as it should;
+    a child killed by a signal (the mutated code faulted) cannot have passed the pin either."""
     assert source.count(old) == 1, "mutation site must be unique: " + what
     mutated = tmp_path / "oracle_mut.cpp"
     mutated.write_text(source.replace(old, new))
     so = tmp_path / "liboracle_mut.so"
     subprocess.check_call(["g++", "-O1", "-std=c++17", "-shared", "-fPIC", "-o", str(so), str(mutated)])
-    lib = C.CDLL(str(so))
-    lib.orc_bruteforce_opt.restype = C.c_longlong
-    lib.orc_bruteforce_best_order.restype = C.c_longlong
-    real = orc.lib()
-    fn = getattr(pins, pin)
-    orc._lib = lib
-    try:
-        with pytest.raises((AssertionError, ValueError)):
-            if pin == "test_example1_tel":
-                for ex in (orc.list_schedule_alg1, orc.list_schedule_rounds):
-                    fn(golden, ex)
-            elif needs_golden:
-                fn(golden)
-            else:
-                fn()
-    finally:
-        orc._lib = real
+    root = os.path.dirname(HERE)
+    r = subprocess.run([sys.executable, "-c", _CHILD, root, str(so), pin, "1" if needs_golden else "0"],
+                       capture_output=True, text=True, timeout=600)
+    assert r.returncode != 3, "the pin %s still passes with: %s" % (pin, what)
+    assert r.returncode == 0 or r.returncode < 0, "child failed unexpectedly (%d): %s" % (r.returncode, r.stderr[-2000:])
