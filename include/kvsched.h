@@ -21,6 +21,10 @@
  *     stream and return without synchronising (sched_sync() waits).
  *   - The caller owns every buffer it passes.  The handle owns device copies of (s, o), the base
  *     order and all scratch memory; sched_destroy() frees them.
+ *   - Device blocks of 1 MiB and more that the library frees (a destroyed handle's snapshots and
+ *     scratch, outgrown staging buffers) are kept in a process-wide per-device cache -- at most
+ *     KVSCHED_POOL_MB MiB in total (environment variable, default 1024, 0 disables the cache) -- and
+ *     reused by later calls; sched_release_cached_memory() returns them to the driver.
  *   - A handle is tied to the CUDA device that was current in sched_init(); calls on one handle
  *     must not overlap in time.
  *   - Arrays are dense, row-major, int32 unless stated; TELs are int64.
@@ -313,6 +317,9 @@ int sched_amin_simulate(int32_t B, int32_t n_max, const int32_t* n_each, const i
 int sched_sorted_f_amin(int32_t n, const int32_t* s, const int32_t* lower, const int32_t* o, int64_t M,
                         int32_t phase1, int32_t* order_out, int32_t* start_out, int64_t* tel_out,
                         int64_t* evictions_out, int64_t* peak_out);
+
+/* Give every cached device block (see "Conventions" above) back to the driver.  Always SCHED_OK. */
+int sched_release_cached_memory(void);
 
 /* Counters since sched_init: kernels launched by this handle, candidates evaluated. */
 int sched_stats(sched_handle h, int64_t* kernel_launches_out, int64_t* evaluations_out);

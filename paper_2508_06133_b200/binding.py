@@ -22,7 +22,7 @@ NBHD_SWAP, NBHD_SWAP_INSERT, NBHD_SAMPLED = 0, 1, 2
 EXPORTS = [
     "sched_init", "sched_init_batch", "sched_set_stream", "sched_sync", "sched_set_prefill_weight", "sched_set_base_order",
     "sched_get_base_order", "sched_eval_batch", "sched_eval_batch_dev", "sched_sweep_dev",
-    "sched_sorted_f", "sched_sorted_f_dev", "sched_sorted_f_local_swap", "sched_sorted_f_local_swap_dev", "sched_sorted_f_dp", "sched_sorted_f_quantile", "sched_online_simulate", "sched_amin_simulate", "sched_sorted_f_amin", "sched_local_search", "sched_accept_move", "sched_last_eval_kernel_ms", "sched_argmin_static_dev", "sched_stats", "sched_destroy",
+    "sched_sorted_f", "sched_sorted_f_dev", "sched_sorted_f_local_swap", "sched_sorted_f_local_swap_dev", "sched_sorted_f_dp", "sched_sorted_f_quantile", "sched_online_simulate", "sched_amin_simulate", "sched_sorted_f_amin", "sched_local_search", "sched_accept_move", "sched_last_eval_kernel_ms", "sched_argmin_static_dev", "sched_release_cached_memory", "sched_stats", "sched_destroy",
     "sched_strerror", "sched_last_cuda_error",
 ]
 
@@ -73,6 +73,7 @@ def load():
     lib.sched_sorted_f_amin.argtypes = [i32, vp, vp, vp, i64, i32, vp, vp, vp, vp, vp]
     lib.sched_local_search.argtypes = [vp, C.c_int, i32, u64, i64, vp, vp, vp, vp]
     lib.sched_accept_move.argtypes = [vp, i64, i64, C.c_int, u64, i32, vp, vp]
+    lib.sched_release_cached_memory.argtypes = []
     lib.sched_stats.argtypes = [vp, vp, vp]
     lib.sched_last_eval_kernel_ms.argtypes = [vp, vp]
     lib.sched_argmin_static_dev.argtypes = [vp, i64, i64, vp, vp]
@@ -281,6 +282,11 @@ class Scheduler:
         _check(load().sched_accept_move(self._h, int(best_tel), int(best_index), 1 if sampled else 0, seed, iteration,
                                         C.byref(acc), C.byref(tel)), "sched_accept_move")
         return bool(acc.value), tel.value
+
+
+def release_cached_memory():
+    """Return the library's cached device blocks to the driver (sched_release_cached_memory)."""
+    _check(load().sched_release_cached_memory(), "sched_release_cached_memory")
 
 
 def argmin_static_dev(tel, best_out, *, count=None, index_base=0, stream=None):

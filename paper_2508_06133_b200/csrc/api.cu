@@ -5,7 +5,9 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <mutex>
 #include <new>
+#include <unordered_map>
 #include <vector>
 
 #include "common.cuh"
@@ -66,25 +68,115 @@ unsigned key_byte_mask(int lo_bits, int hi_bits) {
     return m;
 }
 
+// ------------------------------------------------------------------------------------------------
+// Device-memory cache.  Creating and destroying a handle allocates and frees a few hundred MB (base
+// run snapshots, staging, per-candidate scratch); cudaFree of such blocks was seen to take from 2 ms
+// to more than half a second on a busy machine.  Blocks of at least 1 MiB therefore go back to a
+// process-wide per-device free list (at most KVSCHED_POOL_MB MiB in total, default 1024, 0 turns the
+// cache off) and are handed out again to later requests of similar size.  kv_free() waits for the
+// device first, exactly as cudaFree does, so a cached block is never still in use.
+// sched_release_cached_memory() returns everything to the driver.
+// ------------------------------------------------------------------------------------------------
+struct PoolBlock { void* p; size_t bytes; int device; };
+std::mutex g_pool_mu;
+std::vector<PoolBlock> g_pool_free;
+std::unordered_map<void*, PoolBlock> g_pool_live;
+size_t g_pool_cached = 0;
+const size_t kPoolMinBlock = 1ull << 20;
+
+size_t pool_cap_bytes() {
+    static const size_t cap = [] {
+        const char* e = getenv("KVSCHED_POOL_MB");
+        const long long mb = e ? atoll(e) : 1024;
+        return (size_t)(mb < 0 ? 0 : mb) << 20;
+    }();
+    return cap;
+}
+
+void pool_trim_locked(int device) {             // device < 0: every device
+    for (size_t k = 0; k < g_pool_free.size();) {
+        if (device < 0 || g_pool_free[k].device == device) {
+            cudaFree(g_pool_free[k].p);
+            g_pool_cached -= g_pool_free[k].bytes;
+            g_pool_free[k] = g_pool_free.back();
+            g_pool_free.pop_back();
+        } else {
+            ++k;
+        }
+    }
+}
+
+cudaError_t kv_malloc(void** out, size_t bytes) {
+    *out = nullptr;
+    if (bytes < kPoolMinBlock || pool_cap_bytes() == 0) return cudaMalloc(out, bytes);
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    const size_t want = (bytes + (kPoolMinBlock - 1)) & ~(kPoolMinBlock - 1);
+    std::lock_guard<std::mutex> lock(g_pool_mu);
+    int best = -1;
+    for (size_t k = 0; k < g_pool_free.size(); ++k) {
+        const PoolBlock& b = g_pool_free[k];
+        if (b.device == dev && b.bytes >= want && b.bytes <= 2 * want && (best < 0 || b.bytes < g_pool_free[best].bytes))
+            best = (int)k;
+    }
+    if (best >= 0) {
+        const PoolBlock b = g_pool_free[best];
+        g_pool_free[best] = g_pool_free.back();
+        g_pool_free.pop_back();
+        g_pool_cached -= b.bytes;
+        g_pool_live[b.p] = b;
+        *out = b.p;
+        return cudaSuccess;
+    }
+    e = cudaMalloc(out, want);
+    if (e == cudaErrorMemoryAllocation) {       // give the cached blocks back and try once more
+        cudaGetLastError();
+        pool_trim_locked(dev);
+        e = cudaMalloc(out, want);
+    }
+    if (e == cudaSuccess) g_pool_live[*out] = PoolBlock{*out, want, dev};
+    return e;
+}
+
+void kv_free(void* p) {
+    if (!p) return;
+    std::unique_lock<std::mutex> lock(g_pool_mu);
+    auto it = g_pool_live.find(p);
+    if (it == g_pool_live.end()) { lock.unlock(); cudaFree(p); return; }
+    const PoolBlock b = it->second;
+    g_pool_live.erase(it);
+    if (g_pool_cached + b.bytes > pool_cap_bytes()) { lock.unlock(); cudaFree(p); return; }
+    lock.unlock();
+    int prev = -1;
+    cudaGetDevice(&prev);
+    if (prev != b.device) cudaSetDevice(b.device);
+    cudaDeviceSynchronize();                    // what cudaFree would have waited for
+    if (prev != b.device && prev >= 0) cudaSetDevice(prev);
+    lock.lock();
+    g_pool_free.push_back(b);
+    g_pool_cached += b.bytes;
+}
+
 template <typename T>
 int dev_alloc(T** p, size_t count) {
     *p = nullptr;
     if (count == 0) count = 1;
-    KV_CUDA(cudaMalloc((void**)p, count * sizeof(T)));
+    KV_CUDA(kv_malloc((void**)p, count * sizeof(T)));
     return SCHED_OK;
 }
 
 int ensure_stage(sched_ctx* h, size_t bytes) {
     if (h->stage_cap >= bytes) return SCHED_OK;
-    if (h->d_stage) { cudaFree(h->d_stage); h->d_stage = nullptr; h->stage_cap = 0; }
-    KV_CUDA(cudaMalloc(&h->d_stage, bytes));
+    if (h->d_stage) { kv_free(h->d_stage); h->d_stage = nullptr; h->stage_cap = 0; }
+    KV_CUDA(kv_malloc((void**)&h->d_stage, bytes));
     h->stage_cap = bytes;
     return SCHED_OK;
 }
 
 int ensure_tel(sched_ctx* h, i64 count) {
     if (h->tel_cap >= count) return SCHED_OK;
-    if (h->d_tel) { cudaFree(h->d_tel); h->d_tel = nullptr; h->tel_cap = 0; }
+    if (h->d_tel) { kv_free(h->d_tel); h->d_tel = nullptr; h->tel_cap = 0; }
     KV_TRY(dev_alloc(&h->d_tel, (size_t)count + 2));
     h->tel_cap = count;
     return SCHED_OK;
@@ -126,7 +218,7 @@ void free_ctx(sched_ctx* h) {
                     h->d_keys_a, h->d_keys_b, h->d_vals_a, h->d_vals_b, h->d_prefP, h->d_prefO,
                     h->d_batch_off, h->d_num_batches, h->d_seg_off, h->d_stage, h->d_base_starts,
                     h->d_state, h->d_sort, h->d_k4, h->d_ls};
-    for (void* p : ptrs) if (p) cudaFree(p);
+    for (void* p : ptrs) if (p) kv_free(p);
     if (h->h_pinned) cudaFreeHost(h->h_pinned);
     if (h->ev_k3_begin) cudaEventDestroy(h->ev_k3_begin);
     if (h->ev_k3_end) cudaEventDestroy(h->ev_k3_end);
@@ -295,8 +387,8 @@ unsigned k3_grid(const sched_ctx* h, i64 count) {
 int order_candidates(sched_ctx* h, const MoveSource& src, i64 count) {
     const size_t need = ((size_t)h->n + 1 + 2 * (size_t)count) * sizeof(int) + 256;
     if (h->k4_cap < need) {
-        if (h->d_k4) { cudaFree(h->d_k4); h->d_k4 = nullptr; h->k4_cap = 0; }
-        KV_CUDA(cudaMalloc(&h->d_k4, need));
+        if (h->d_k4) { kv_free(h->d_k4); h->d_k4 = nullptr; h->k4_cap = 0; }
+        KV_CUDA(kv_malloc((void**)&h->d_k4, need));
         h->k4_cap = need;
     }
     int* bins = (int*)h->d_k4;
@@ -495,8 +587,8 @@ int sched_eval_batch_dev(sched_handle h, int kind, int64_t count, const void* ca
         // ids of every candidate by ascending (start, id): K1 with one segment per candidate
         const size_t need = (size_t)total * (2 * sizeof(u64) + 2 * sizeof(int)) + (size_t)(count + 1) * sizeof(int) + 64;
         if (h->sort_cap < need) {
-            if (h->d_sort) { cudaFree(h->d_sort); h->d_sort = nullptr; h->sort_cap = 0; }
-            KV_CUDA(cudaMalloc(&h->d_sort, need));
+            if (h->d_sort) { kv_free(h->d_sort); h->d_sort = nullptr; h->sort_cap = 0; }
+            KV_CUDA(kv_malloc((void**)&h->d_sort, need));
             h->sort_cap = need;
         }
         u64* ka = (u64*)h->d_sort; u64* kb = ka + total;
@@ -731,10 +823,10 @@ static int phase1_dp(sched_handle h) {
 #undef DP_CUDA
     } while (0);
     cudaStreamSynchronize(st);
-    if (dpA) cudaFree(dpA);
-    if (dpB) cudaFree(dpB);
-    if (took) cudaFree(took);
-    if (small) cudaFree(small);
+    if (dpA) kv_free(dpA);
+    if (dpB) kv_free(dpB);
+    if (took) kv_free(took);
+    if (small) kv_free(small);
     return rc;
 }
 
@@ -1000,8 +1092,8 @@ int sched_online_simulate(int32_t B, int32_t n_max, const int32_t* n_each, const
     if (e0) cudaEventDestroy(e0);
     if (e1) cudaEventDestroy(e1);
     int* frees[] = {d_n, d_a, d_s, d_o, d_start, d_status};
-    for (int* ptr : frees) if (ptr) cudaFree(ptr);
-    if (d_lat) cudaFree(d_lat);
+    for (int* ptr : frees) if (ptr) kv_free(ptr);
+    if (d_lat) kv_free(d_lat);
     return rc;
 }
 
@@ -1094,8 +1186,8 @@ static int amin_run(int32_t B, int32_t n_max, const int32_t* n_each, const int32
     if (e0) cudaEventDestroy(e0);
     if (e1) cudaEventDestroy(e1);
     int* frees[] = {d_n, d_s, d_l, d_o, d_ord, d_start, d_status};
-    for (int* ptr : frees) if (ptr) cudaFree(ptr);
-    if (d_res) cudaFree(d_res);
+    for (int* ptr : frees) if (ptr) kv_free(ptr);
+    if (d_res) kv_free(d_res);
     return rc;
 }
 
@@ -1126,6 +1218,12 @@ int sched_sorted_f_amin(int32_t n, const int32_t* s, const int32_t* lower, const
         rc = amin_run(1, n, &n, s, lower, o, M, nullptr, h->d_order, start_out, tel_out, evictions_out, peak_out, nullptr);
     sched_destroy(h);
     return rc;
+}
+
+int sched_release_cached_memory(void) {
+    std::lock_guard<std::mutex> lock(g_pool_mu);
+    pool_trim_locked(-1);
+    return SCHED_OK;
 }
 
 int sched_stats(sched_handle h, int64_t* kernel_launches_out, int64_t* evaluations_out) {

@@ -722,6 +722,35 @@ def test_sharded_search_driver_on_one_gpu_equals_the_library_search():
         assert e.value.code == kv.E_INVAL
 
 
+def test_cached_device_memory_is_reused_and_released():
+    """Handles created and destroyed in a row take their large blocks from the library's cache (stale
+    contents must not matter: every result is again the oracle's), and
+    sched_release_cached_memory gives the blocks back to the driver."""
+    import torch
+    inst = W.mixed_1k()
+    n = inst.n
+    total = n * (n - 1) // 2 + n * (n - 1)
+    r_order, _ = orc.sorted_f_prefix(inst.s, inst.o, inst.M)
+    seen = []
+    for rep in range(3):
+        codes = (W.u64(300 + rep, 0, np.arange(500)) % np.uint64(total)).astype(np.int64)
+        with kv.Scheduler(inst.s, inst.o, inst.M) as h:
+            order, offs, tel = h.sorted_f()
+            tels, _, _ = h.eval_batch(kv.CAND_MOVE, codes)
+        assert (order == r_order).all()
+        assert (tels == oracle_moves(inst.s, inst.o, inst.M, r_order, codes)).all()
+        seen.append(tel)
+    assert len(set(seen)) == 1
+    torch.cuda.synchronize()
+    free_cached = torch.cuda.mem_get_info()[0]
+    kv.release_cached_memory()
+    free_released = torch.cuda.mem_get_info()[0]
+    assert free_released >= free_cached + (4 << 20)          # the 1,000-request snapshots alone are 4 MB
+    kv.release_cached_memory()                               # nothing left: still fine
+    with kv.Scheduler(inst.s, inst.o, inst.M) as h:
+        assert h.sorted_f()[2] == seen[0]
+
+
 def test_device_pointer_candidates_are_bounds_checked_on_the_device():
     import torch
     dev = torch.device("cuda", torch.cuda.current_device())
