@@ -203,7 +203,10 @@ def main():
         raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
-    if world > 1:
+    # under torchrun (RANK set) the process group is used even with one rank, so that the very same
+    # barrier / max-over-ranks path runs at every N
+    multi = "RANK" in os.environ and "MASTER_ADDR" in os.environ
+    if multi:
         dist.init_process_group("nccl", device_id=dev)
 
     n, sum_o = inst.n, int(inst.o.sum())
@@ -232,7 +235,7 @@ def main():
     h.sync()
     launches0, _ = h.stats()
     sampler = ClockSampler(local_rank)
-    if world > 1:
+    if multi:
         dist.barrier()
     torch.cuda.synchronize()
     sampler.start()
@@ -243,12 +246,12 @@ def main():
         kern_ms.append(b)
     torch.cuda.synchronize()
     clocks = sampler.stop()
-    if world > 1:
+    if multi:
         dist.barrier()
     h.sync()
     launches1, _ = h.stats()
     total_ms = float(sum(step_ms))
-    if world > 1:
+    if multi:
         total_ms = max_over_ranks(total_ms, dist, dev)
     value = world * count * args.steps / (total_ms * 1e-3)
 
@@ -303,7 +306,7 @@ def main():
         hh.close()
         return res
     e2e_step(e2e_steps)
-    if world > 1:
+    if multi:
         dist.barrier()
     torch.cuda.synchronize()
     t0 = time.perf_counter()
@@ -311,7 +314,7 @@ def main():
         e2e_step(k)
     torch.cuda.synchronize()
     dt = time.perf_counter() - t0
-    if world > 1:
+    if multi:
         dt = max_over_ranks(dt, dist, dev)
     e2e = {"value": world * count * e2e_steps / dt, "unit": "evals/s",
            "h2d_bytes_per_step": int(8 * n + 8 * count), "d2h_bytes_per_step": int(8 * count + 4 * n + 8),
@@ -356,7 +359,7 @@ def main():
         }
         print(json.dumps(out))
     h.close()
-    if world > 1:
+    if multi:
         dist.destroy_process_group()
 
 
