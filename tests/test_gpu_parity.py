@@ -710,6 +710,21 @@ def test_sharded_search_driver_on_one_gpu_equals_the_library_search():
                 assert (best[1], best[0]) == tuple(r_trace[it])
                 ev.accept(best[0], best[1], nbhd == kv.NBHD_SAMPLED, 3, it)
             assert (h.get_base_order() == r_order).all()
+    # the exchange itself over NCCL (one rank: the same calls every rank of a larger job makes)
+    import os
+    import torch
+    import torch.distributed as dist
+    dist.init_process_group("nccl", init_method="tcp://127.0.0.1:%d" % (29600 + os.getpid() % 300), rank=0, world_size=1,
+                            device_id=torch.device("cuda", 0))
+    try:
+        r_order, r_tel, r_done, r_trace = orc.local_search(s, o, M, kv.NBHD_SAMPLED, 6, start, seed=8, samples=150)
+        with kv.Scheduler(s, o, M) as h:
+            h.set_base_order(start)
+            tel, done, trace = par.sharded_local_search(par.GpuEvaluator(h), kv.NBHD_SAMPLED, 6, seed=8, samples_per_iter=150,
+                                                        comm=par.TorchComm(device=torch.device("cuda", 0)))
+            assert (tel, done) == (r_tel, r_done) and (trace == r_trace).all() and (h.get_base_order() == r_order).all()
+    finally:
+        dist.destroy_process_group()
     with kv.Scheduler(s, o, M) as h:
         h.set_base_order(start)
         base = orc.list_schedule_rounds(s, o, M, start)[1]
