@@ -183,7 +183,7 @@ def main():
     ap.add_argument("--moves", type=int, default=1 << 22, help="sampled moves evaluated per step and GPU")
     ap.add_argument("--ref-moves", type=int, default=96, help="moves per step of the CPU reference arm")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="mixed_10k", choices=["mixed_10k", "mixed_1k", "paper_scale"])
+    ap.add_argument("--workload", default="mixed_10k", choices=["mixed_10k", "mixed_1k", "paper_scale", "heavy_100k"])
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="budget of the cpu_baseline leg")
     args = ap.parse_args()
 
