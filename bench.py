@@ -36,7 +36,7 @@ SMEM_BYTES_PER_CLK_PER_SM = 128          # shared-memory bandwidth of one SM (pr
 INT_OPS_PER_CLK_PER_SM = 64              # 32-bit integer adds per clock and SM (probe: 63.7)
 FALLBACK_HBM_GBS, FALLBACK_SM_MHZ = 6650.0, 1965.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one simulator launch, from a one-pass ncu capture of
-# this very launch (profiles/k3_eval_moves_mixed_n10000_dram_traffic.md); keyed by (workload, moves per
+# this very launch (summary under profiles/); keyed by (workload, moves per
 # launch, simulator source files' digest) so that it turns into null when the kernel changes
 K3_TRAFFIC = {("mixed_n10000", 1 << 22): (60.61e6 + 11.38e6, "21db94945fc6e5e0")}
 
