@@ -29,8 +29,8 @@
 //   While the head of the queue is refused nothing is admitted and occ only grows, so the bound on
 //   its wait that the window test gives (a cell over budget by x at offset r needs min(x, r+1) more
 //   rounds) stays valid until the next eviction.  Rounds in which nothing can happen (no overflow;
-//   head still bound to wait, or not even its first round fits) are walked by one thread, a handful
-//   of instructions each.
+//   head still bound to wait, or not even its first round fits) are walked by one warp, 32 rounds
+//   per step (the running aggregates of a round are prefix sums of the event cells).
 #pragma once
 
 #include "common.cuh"
@@ -158,26 +158,55 @@ __global__ void __launch_bounds__(K7_THREADS) k7_amin(const AminParams P) {
 
     for (i64 turn = 0;; ++turn) {
         if (turn > turn_cap) { failed = true; break; }
-        if (tid == 0) {
-            // rounds in which nothing can be decided: step 1 only
+        if (tid < 32) {
+            // rounds in which nothing can be decided (step 1 only), 32 at a time: lane l takes round
+            // t + l.  A round reads only its own cells and the running (cnt, A, remaining), which are
+            // prefix sums of the event cells, so the 32 rounds are evaluated together and the walk
+            // stops at the first lane whose round needs the whole CTA (or ends the run).
+            const int lane = tid;
             int act = K7_ACT_WORK;
             const int head_s = head < n ? ps[head] : 0;
             for (;;) {
-                const int k = t & mask;
-                cnt += (unsigned)dc[k]; A += dA[k]; remaining -= fin[k];
-                dc[k] = 0; dA[k] = 0u; fin[k] = 0;
-                const int u = occ[k] + (int)(A + cnt * (unsigned)t);
-                occ[k] = u;
-                if (remaining == 0) { act = K7_ACT_DONE; break; }
+                const int tau = t + lane;
+                const int k = tau & mask;
+                int cs = dc[k];
+                unsigned as = dA[k];
+                int fs = fin[k];
+                const int oc = occ[k];
+#pragma unroll
+                for (int d = 1; d < 32; d <<= 1) {
+                    const int c2 = __shfl_up_sync(KV_FULL, cs, d);
+                    const unsigned a2 = __shfl_up_sync(KV_FULL, as, d);
+                    const int f2 = __shfl_up_sync(KV_FULL, fs, d);
+                    if (lane >= d) { cs += c2; as += a2; fs += f2; }
+                }
+                const unsigned cnt_l = cnt + (unsigned)cs, A_l = A + as;
+                const int rem_l = remaining - fs;
+                const int u = oc + (int)(A_l + cnt_l * (unsigned)tau);
+                const bool done = rem_l == 0;
                 // the head's first round is the current one: if it does not fit there, the window
                 // test cannot succeed in this iteration and the CTA need not be woken for it
-                if (u > M || (head < n && t >= t_ok && u + head_s + 1 <= M)) break;
-                if ((i64)t >= round_cap) { act = K7_ACT_CAP; break; }
-                peak = max(peak, u);
-                occ[k] = 0;
-                ++t;
+                const bool work = u > M || (head < n && tau >= t_ok && u + head_s + 1 <= M);
+                const bool cap = (i64)tau >= round_cap;
+                const unsigned stops = __ballot_sync(KV_FULL, done || work || cap);
+                const int first = stops ? __ffs(stops) - 1 : 32;
+                if (lane <= first) { dc[k] = 0; dA[k] = 0u; fin[k] = 0; }          // events consumed
+                if (lane < first) occ[k] = 0;                                        // a round that is over
+                else if (lane == first) occ[k] = u;
+                peak = max(peak, kv_warp_max(lane < first ? u : 0));
+                const int src = first < 32 ? first : 31;
+                cnt = __shfl_sync(KV_FULL, cnt_l, src);
+                A = __shfl_sync(KV_FULL, A_l, src);
+                remaining = __shfl_sync(KV_FULL, rem_l, src);
+                if (first < 32) {
+                    t += first;
+                    const int why = done ? K7_ACT_DONE : (work ? K7_ACT_WORK : K7_ACT_CAP);
+                    act = __shfl_sync(KV_FULL, why, first);
+                    break;
+                }
+                t += 32;
             }
-            ctl.t = t; ctl.remaining = remaining; ctl.peak = peak; ctl.act = act; ctl.cnt = cnt; ctl.A = A;
+            if (lane == 0) { ctl.t = t; ctl.remaining = remaining; ctl.peak = peak; ctl.act = act; ctl.cnt = cnt; ctl.A = A; }
         }
         __syncthreads();
         t = ctl.t; remaining = ctl.remaining; peak = ctl.peak; cnt = ctl.cnt; A = ctl.A;
