@@ -8,7 +8,7 @@
  * TEL = sum_i c_i, in rounds.
  *
  * An ORDER (a permutation of the requests) is turned into start times by Phase 2 of Algorithm 1
- * (Appendix C): every round, finished requests leave, then pending requests are admitted in list
+ * (the supplement to Section 3): every round, finished requests leave, then pending requests are admitted in list
  * order for as long as the memory of all running requests stays within M at every future round;
  * the first request that does not fit ends that round's admissions.
  *
@@ -58,7 +58,7 @@ enum {
     SCHED_CAND_POLICY = 3        /* int32[count]: SCHED_POLICY_* ids; each instance x each policy        */
 };
 
-/* Order policies (Section 2.3, Appendix A, Section 7). Ties always go to the lower request index. */
+/* Order policies (Section 2.3, the supplement to Section 2, Section 7). Ties always go to the lower request index. */
 enum {
     SCHED_POLICY_FCFS = 0,        /* index order                                                         */
     SCHED_POLICY_SOF = 1,         /* shortest output first (MC-SF): ascending o                          */
@@ -99,7 +99,7 @@ int sched_sync(sched_handle h);
 /* Prefill weight of the batch metric (Section 7, "Robustness to prefill weighting"):
  * G(X) = sum (alpha * s_i + o_i) / |X|^2 with alpha = alpha_num / alpha_den; alpha = 0 (the default,
  * 0/1) is the F-metric.  Applies to the following sched_sorted_f() and sched_sorted_f_local_swap()
- * calls of this handle (in Algorithm 4 a swap then improves iff alpha*s_in + o_in < alpha*s_out +
+ * calls of this handle (in Algorithm 3 a swap then improves iff alpha*s_in + o_in < alpha*s_out +
  * o_out); the exact DP and the POLICY candidates keep F.  Compared exactly on integer weights.
  * SCHED_E_INVAL unless 0 <= alpha_num <= 2^20 and 1 <= alpha_den <= 2^20. */
 int sched_set_prefill_weight(sched_handle h, int32_t alpha_num, int32_t alpha_den);
@@ -132,14 +132,17 @@ int sched_eval_batch_dev(sched_handle h, int kind, int64_t count, const void* ca
 /* Evaluate the contiguous move-code range [first_code, first_code + count) (SWAP_INSERT coding)
  * against the base order, or -- if sampled != 0 -- the sampled moves m = first_code .. first_code +
  * count - 1 of iteration `iteration` under `seed`; then reduce to the best (TEL, index) pair.
- *   tel_out  : device int64[count], nullable (per-candidate TELs are still reduced if NULL).
+ *   tel_out  : device int64[count], nullable (per-candidate TELs are still reduced if NULL); any
+ *              8-byte aligned address will do (e.g. a slice of a larger array).
  *   best_out : device int64[2] = {min TEL, lowest index (code or m) attaining it}.
- * Asynchronous on the handle's stream.  This is one neighbourhood sweep of sched_local_search(). */
+ * Asynchronous on the handle's stream.  This is one neighbourhood sweep of sched_local_search().
+ * SCHED_E_INVAL (nothing is launched): batch handle, n < 2, count <= 0, a range that leaves the
+ * neighbourhood, best_out NULL, or tel_out / best_out not 8-byte aligned. */
 int sched_sweep_dev(sched_handle h, int sampled, uint64_t seed, int32_t iteration,
                     int64_t first_code, int64_t count, int64_t* tel_out, int64_t* best_out);
 
 /* Sorted-F (Algorithm 1 Phase 1 + Phase 2) with prefix-F batch selection: requests are sorted by
- * (s+o, o, index) ascending -- the order Algorithm 4 starts from; from the current offset a, with
+ * (s+o, o, index) ascending -- the order Algorithm 3 starts from; from the current offset a, with
  * k_max the longest prefix of the remaining requests whose sum(s+o) <= M, the batch is the prefix
  * of length k* = argmin_{1<=k<=k_max} (sum of o over the prefix) / k^2, ties to the larger k
  * (Section 3: minimise F, prefer the larger batch; compared exactly in integers); the batch is
@@ -155,7 +158,7 @@ int sched_sorted_f(sched_handle h, int32_t* order_out, int32_t* batch_offsets_ou
 int sched_sorted_f_dev(sched_handle h, int32_t* order_out, int32_t* batch_offsets_out,
                        int32_t* num_batches_out, int64_t* tel_out);
 
-/* Sorted-F with Algorithm 4 (Local Swap Search, Section 5.2 and Appendix D) as the Phase-1 solver --
+/* Sorted-F with Algorithm 3 (Local Swap Search, Section 5.2 and the supplement to Section 5) as the Phase-1 solver --
  * the variant the paper's experiments use at n = 2000.  Repeat on the requests not yet placed:
  * sort by ascending s+o (ties: lower index); first-fit fill up to sum(s+o) <= M; then, walking
  * r_out over the batch (insertion order; a swapped-in request takes the replaced one's place) and
@@ -170,7 +173,7 @@ int sched_sorted_f_local_swap(sched_handle h, int32_t* order_out, int32_t* batch
 int sched_sorted_f_local_swap_dev(sched_handle h, int32_t* order_out, int32_t* batch_offsets_out,
                                   int32_t* num_batches_out, int64_t* tel_out);
 
-/* Sorted-F with Algorithm 5 (Quantile Greedy Selection, Section 5.3 and Appendix D) as the Phase-1
+/* Sorted-F with Algorithm 4 (Quantile Greedy Selection, Section 5.3 and the supplement to Section 5) as the Phase-1
  * solver: repeat on the requests not yet placed { walk them in ascending (o, index); draw a sample
  * of max(1, floor(m/2)) of the m requests; Q_p, Q_o = 0.3-quantiles of s+o and of o over the sample;
  * pass 1 admits, in walking order, every request with s+o <= Q_p, o <= Q_o that still fits in M;
@@ -185,7 +188,7 @@ int sched_sorted_f_local_swap_dev(sched_handle h, int32_t* order_out, int32_t* b
 int sched_sorted_f_quantile(sched_handle h, uint64_t seed, int32_t* order_out, int32_t* batch_offsets_out,
                             int32_t* num_batches_out, int64_t* tel_out);
 
-/* Sorted-F with Algorithm 2 (exact dynamic programme, Section 5.1 and Appendix D) as the Phase-1
+/* Sorted-F with Algorithm 2 (exact dynamic programme, Section 5.1 and the supplement to Section 5) as the Phase-1
  * solver: repeat on the requests not yet placed { dp[k][m] = min sum of o over k-subsets whose
  * sum(s+o) is exactly m <= M, requests taken in ascending index, a cell replaced only by a strictly
  * smaller value; the batch is the cell minimising dp/k^2, ties to the larger k (Section 3), then the
@@ -268,7 +271,7 @@ int sched_argmin_static_dev(const int64_t* tel, int64_t count, int64_t index_bas
  *       planned again when it has never been planned, `period` iterations after the last plan, when
  *       it had run empty, or when the arrivals since the last plan reach half of the backlog size at
  *       that plan.  A plan sorts the pending requests by ascending (s+o, index), orders the first
- *       `lookahead` of them by Sorted-F with Algorithm 4 (every batch by ascending (o, index)) and
+ *       `lookahead` of them by Sorted-F with Algorithm 3 (every batch by ascending (o, index)) and
  *       appends the others in sorted order.  The paper uses period = 10, lookahead = 300.
  * start_out [B, n_max] receives the start times (-1 where a row has no request), latency_out [B] the
  * sum of (p + o - arrival) per stream; kernel_ms_out (nullable) the device time of the simulation.
@@ -281,7 +284,7 @@ int sched_online_simulate(int32_t B, int32_t n_max, const int32_t* n_each, const
                           int32_t lookahead, int32_t* start_out, int64_t* latency_out, float* kernel_ms_out);
 
 /* Sorted-F + A_min, Phase 2 (Section 5.5, "Handling Prediction Uncertainty via Adaptive Output Length
- * Refinement"; Algorithm 6 in Appendix D): B independent scenarios executed to completion when only a
+ * Refinement"; Algorithm 5 in the supplement to Section 5): B independent scenarios executed to completion when only a
  * lower bound lower[i] <= o[i] of every decode length is known to the scheduler, one CTA per scenario.
  * Scenario b has n_each[b] <= n_max requests in row b of the [B, n_max] arrays s / lower / o / order
  * (entries past n_each[b] are ignored); order is the list to execute, a permutation of 0..n_each[b]-1
@@ -308,8 +311,8 @@ int sched_amin_simulate(int32_t B, int32_t n_max, const int32_t* n_each, const i
                         const int32_t* o, int64_t M, const int32_t* order, int32_t* start_out, int64_t* tel_out,
                         int64_t* evictions_out, int64_t* peak_out, float* kernel_ms_out);
 
-/* Sorted-F + A_min end to end for one backlog (Algorithm 6): Phase 1 of Sorted-F on (s, lower) --
- * phase1 = 0: prefix-F batch selection as in sched_sorted_f(); 1: Algorithm 4 as in
+/* Sorted-F + A_min end to end for one backlog (Algorithm 5): Phase 1 of Sorted-F on (s, lower) --
+ * phase1 = 0: prefix-F batch selection as in sched_sorted_f(); 1: Algorithm 3 as in
  * sched_sorted_f_local_swap() -- then the executor of sched_amin_simulate() on the resulting list.
  *   order_out : host int32[n], nullable, the Phase-1 list.  Other outputs as above with B = 1.
  * Host pointers; creates and destroys a handle internally.  Errors as sched_init() and
@@ -317,6 +320,48 @@ int sched_amin_simulate(int32_t B, int32_t n_max, const int32_t* n_each, const i
 int sched_sorted_f_amin(int32_t n, const int32_t* s, const int32_t* lower, const int32_t* o, int64_t M,
                         int32_t phase1, int32_t* order_out, int32_t* start_out, int64_t* tel_out,
                         int64_t* evictions_out, int64_t* peak_out);
+
+/* Peak rates of the execution resources that bound the schedule simulator, measured on the current
+ * CUDA device by short probe kernels (measurement support for rooflines; the paper has no
+ * counterpart).  Each probe keeps every SM busy with independent dependency chains of one kind of
+ * work and is timed with CUDA events on `cuda_stream` (cudaStream_t as void*, NULL: default stream);
+ * the best of `repeats` (1..64) timed launches after one warm-up launch is reported, in lane
+ * operations per second (32 per warp instruction) or bytes per second, at whatever clock the device
+ * runs while probed:
+ *   out[SCHED_PROBE_INT_ADD]      32-bit integer adds
+ *   out[SCHED_PROBE_INT_ADD_MAX]  adds and maxima alternating
+ *   out[SCHED_PROBE_INT_MAD]      32-bit integer multiply-adds
+ *   out[SCHED_PROBE_SIM_MIX]      the simulator's window-pass mix: multiply-add, 3-input max, add
+ *   out[SCHED_PROBE_SMEM_LOAD]    shared-memory loads, 16 bytes per thread and access
+ *   out[SCHED_PROBE_SMEM_STORE]   shared-memory stores, 16 bytes per thread and access
+ *   out[SCHED_PROBE_INT_ALU]      maxima and exclusive-ors alternating: work that only the integer
+ *                                 ALU pipe executes (the compiler may spread plain adds over the
+ *                                 ALU and the multiply-add pipe, never these)
+ *   out : host double[n_out], n_out >= SCHED_PROBE_COUNT.
+ * Synchronous; allocates and frees a few MB of device memory; about 50 ms on one GPU.
+ * SCHED_E_INVAL: NULL out, n_out too small, repeats out of range. */
+enum {
+    SCHED_PROBE_INT_ADD = 0,
+    SCHED_PROBE_INT_ADD_MAX = 1,
+    SCHED_PROBE_INT_MAD = 2,
+    SCHED_PROBE_SIM_MIX = 3,
+    SCHED_PROBE_SMEM_LOAD = 4,
+    SCHED_PROBE_SMEM_STORE = 5,
+    SCHED_PROBE_INT_ALU = 6,
+    SCHED_PROBE_COUNT = 7
+};
+int sched_probe_peaks(double* out, int32_t n_out, int32_t repeats, void* cuda_stream);
+
+/* Test support (the paper has no counterpart): every device loop of this library whose trip count
+ * depends on the data is bounded by a cap that it can never reach on valid input; a loop that does
+ * reach its cap records that in a status word and returns, the kernel ends normally, and the host
+ * call that reads the status (the host-pointer entry points, sched_sync, sched_local_search,
+ * sched_accept_move) returns SCHED_E_INTERNAL and clears it.  This call lowers every such cap on the
+ * current CUDA device to `cap` iterations so that a test can make one run out (cap = 0: the first
+ * request that has to wait gives up); a negative cap restores the natural bounds.  Results computed
+ * while a lowered cap is in force are meaningless.  Synchronises the device; not for concurrent use
+ * with running kernels of this library. */
+int sched_debug_set_loop_cap(int32_t cap);
 
 /* Give every cached device block (see "Conventions" above) back to the driver.  Always SCHED_OK. */
 int sched_release_cached_memory(void);

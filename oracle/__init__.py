@@ -26,7 +26,7 @@ SWAP, SWAP_INSERT, SAMPLED = 0, 1, 2
 def build(force: bool = False) -> str:
     if force or not os.path.exists(_SO) or os.path.getmtime(_SO) < os.path.getmtime(_SRC):
         tmp = _SO + ".%d.tmp" % os.getpid()
-        subprocess.check_call(["g++", "-O2", "-std=c++17", "-shared", "-fPIC", "-o", tmp, _SRC])
+        subprocess.check_call(["g++", "-O2", "-std=c++17", "-pthread", "-shared", "-fPIC", "-o", tmp, _SRC])
         os.replace(tmp, _SO)
     return _SO
 
@@ -169,6 +169,19 @@ def eval_moves(s, o, M, base, types, mi, mj):
     return tel
 
 
+def eval_moves_threads(s, o, M, base, types, mi, mj, threads=1, literal=False):
+    """``eval_moves`` with the candidates split over ``threads`` host threads (CPU-baseline timing);
+    ``literal`` scores with Algorithm 1 Phase 2 as listed instead of the per-round form."""
+    s, o, base = _i32(s), _i32(o), _i32(base)
+    types, mi, mj = _i32(types), _i32(mi), _i32(mj)
+    tel = np.zeros(len(types), dtype=np.int64)
+    rc = lib().orc_eval_moves_threads(len(s), _p(s), _p(o), C.c_longlong(M), _p(base), C.c_longlong(len(types)),
+                                      _p(types), _p(mi), _p(mj), _p(tel), int(threads), 1 if literal else 0)
+    if rc != 0:
+        raise ValueError("invalid instance")
+    return tel
+
+
 def local_search(s, o, M, neighbourhood, iters, order, seed=0, samples=0):
     """Returns (final order, TEL, iterations done, trace[(code, best TEL)] per iteration)."""
     s, o = _i32(s), _i32(o)
@@ -199,7 +212,7 @@ def bruteforce_best_order(s, o, M):
 
 
 def local_swap_batch(ids, s, o, M):
-    """Algorithm 4 on the request set ``ids``.  Returns (X in walking order, accepted swaps)."""
+    """Algorithm 3 on the request set ``ids``.  Returns (X in walking order, accepted swaps)."""
     s, o, ids = _i32(s), _i32(o), _i32(ids)
     chosen = np.zeros(len(ids), dtype=np.int32)
     sw = C.c_longlong(0)
@@ -210,7 +223,7 @@ def local_swap_batch(ids, s, o, M):
 
 
 def sorted_f_local_swap(s, o, M):
-    """Sorted-F with Algorithm 4 as Phase-1 solver.  Returns (order, batch offsets, accepted swaps)."""
+    """Sorted-F with Algorithm 3 as Phase-1 solver.  Returns (order, batch offsets, accepted swaps)."""
     s, o = _i32(s), _i32(o)
     n = len(s)
     order = np.zeros(n, dtype=np.int32)
@@ -239,12 +252,12 @@ def sorted_g_prefix(s, o, M, a_num, a_den):
 
 
 def sorted_g_local_swap(s, o, M, a_num, a_den):
-    """Sorted-G with Algorithm 4 as the batch solver."""
+    """Sorted-G with Algorithm 3 as the batch solver."""
     return _sorted_g(lib().orc_sorted_g_local_swap, s, o, M, a_num, a_den)
 
 
 def quantile_greedy_batch(ids, s, o, M, sample):
-    """Algorithm 5 on the request set ``ids`` with the given sample.
+    """Algorithm 4 on the request set ``ids`` with the given sample.
     Returns (X in admission order, Q_p, Q_o)."""
     s, o, ids, sample = _i32(s), _i32(o), _i32(ids), _i32(sample)
     chosen = np.zeros(len(ids), dtype=np.int32)
@@ -257,7 +270,7 @@ def quantile_greedy_batch(ids, s, o, M, sample):
 
 
 def quantile_sample(ids, o, seed, batch):
-    """The reproducible 'random subset' of Algorithm 5 for batch number ``batch``."""
+    """The reproducible 'random subset' of Algorithm 4 for batch number ``batch``."""
     o, ids = _i32(o), _i32(ids)
     out = np.zeros(max(1, len(ids)), dtype=np.int32)
     c = lib().orc_quantile_sample(len(ids), _p(ids), _p(o), C.c_uint64(seed), int(batch), _p(out))
@@ -265,7 +278,7 @@ def quantile_sample(ids, o, seed, batch):
 
 
 def sorted_f_quantile(s, o, M, seed):
-    """Sorted-F with Algorithm 5 as Phase-1 solver.  Returns (order, batch offsets)."""
+    """Sorted-F with Algorithm 4 as Phase-1 solver.  Returns (order, batch offsets)."""
     s, o = _i32(s), _i32(o)
     n = len(s)
     order = np.zeros(n, dtype=np.int32)
@@ -298,7 +311,7 @@ def online_schedule(a, s, o, M, policy, period=10, lookahead=300):
 
 
 def amin_schedule(s, lower, o, M, order):
-    """Phase 2 of Sorted-F + A_min (Algorithm 6) on the given list with lower bounds ``lower`` of the
+    """Phase 2 of Sorted-F + A_min (Algorithm 5) on the given list with lower bounds ``lower`` of the
     decode lengths.  Returns (final start times, TEL, evictions, peak memory actually used)."""
     s, lower, o, order = _i32(s), _i32(lower), _i32(o), _i32(order)
     n = len(s)

@@ -3,10 +3,10 @@
 // A plain, slow, single-threaded restatement of what the paper defines: the memory model and
 // total end-to-end latency (Section 2.1-2.2, integer program of Section 6.1), the F-metric and
 // Sorted-F (Section 3, Algorithm 1), the exact dynamic programme (Section 5.1, Algorithm 2),
-// Local Swap Search and Quantile Greedy Selection (Sections 5.2-5.3, Algorithms 4 and 5),
+// Local Swap Search and Quantile Greedy Selection (Sections 5.2-5.3, Algorithms 3 and 4),
 // Sorted-G (Section 7), the online policies of Section 6.2 (FCFS, shortest decode first and
 // Sorted-F-Online under arrivals over time), the executor of Sorted-F + A_min under lower-bound
-// predictions (Section 5.5, Algorithm 6), and
+// predictions (Section 5.5, Algorithm 5), and
 // an order-level local search that scores every neighbour with Algorithm 1's Phase 2.  It exists
 // so that the GPU library can be checked against it; it shares no code with that library, is never
 // called by it, and nothing here is tuned for speed.  All arithmetic is integer.
@@ -19,18 +19,19 @@
 //
 // Parity status: every function below is pinned by tests that do not go through this file's own
 // formulas (paper's worked example, closed forms, brute force), except where marked
-// "parity unpinned".  O12 (Algorithm 5): the routine is pinned for a GIVEN sample (hand-worked
+// "parity unpinned".  O12 (Algorithm 4): the routine is pinned for a GIVEN sample (hand-worked
 // cases, a library quantile, maximality), and the sampling hash to the generator's published
 // values; but which subset "random subset" means and how the 0.3-quantile of a finite sample is
 // read are choices no printed value fixes -- for those two choices: parity unpinned.  O13 (online
-// arrivals) and O14 (Algorithm 6): the executors are pinned (reductions to the offline executor,
+// arrivals) and O14 (Algorithm 5): the executors are pinned (reductions to the offline executor,
 // feasibility, hand-worked cases); which requests an online plan covers and where arrivals go, and
-// for Algorithm 6 where an evicted request re-enters the queue and how equal estimates are
+// for Algorithm 5 where an evicted request re-enters the queue and how equal estimates are
 // ordered, are readings no printed value fixes -- for those choices: parity unpinned.
 #include <algorithm>
 #include <cstdint>
 #include <cstring>
 #include <numeric>
+#include <thread>
 #include <vector>
 
 typedef long long i64;
@@ -158,7 +159,7 @@ int orc_list_schedule_rounds(int n, const int* s, const int* o, i64 M, const int
 
 // ---------------------------------------------------------------------------------------------
 // O3. Order policies.  0 = FCFS (index order, Section 7), 1 = shortest output first (MC-SF,
-//     Section 2.3), 2 = smallest s+o first (MC-SF_2, Appendix A).  Ties: lower index first.
+//     Section 2.3), 2 = smallest s+o first (MC-SF_2, the supplement to Section 2).  Ties: lower index first.
 // ---------------------------------------------------------------------------------------------
 void orc_policy_order(int n, const int* s, const int* o, int policy, int* order) {
     std::iota(order, order + n, 0);
@@ -184,7 +185,7 @@ int orc_f_compare(i64 sumA, i64 kA, i64 sumB, i64 kB) {
 // O4. Exact Phase 1 by enumeration of all non-empty subsets of `ids` (m <= 24).
 //     reading 0: Algorithm 1's constraint  M(X, o_j) <= M for all j in X  with all of X started
 //                together, i.e. sum_{i in X, o_i >= o_j} (s_i + o_j) <= M;
-//     reading 1: sum (s_i + o_i) <= M, the constraint Algorithms 2, 4 and 5 use.
+//     reading 1: sum (s_i + o_i) <= M, the constraint Algorithms 2, 3 and 4 use.
 //     Minimise (F, -|X|); then smaller sum(s+o); then the lexicographically smallest index list.
 // Writes the chosen members (ascending position in `ids`) and returns their count.
 // ---------------------------------------------------------------------------------------------
@@ -230,54 +231,57 @@ int orc_phase1_enumerate(int m, const int* ids, const int* s, const int* o, i64 
 }
 
 // ---------------------------------------------------------------------------------------------
-// O5. Algorithm 2 (exact dynamic programme), as printed: dp[k][m] = min sum of o over k-subsets
-//     whose sum(s+o) is exactly m; requests taken one at a time, k descending, strict '<' update;
-//     path[k][m] kept as a bit set (m <= 128 requests).  The final scan follows Section 3's tie
-//     rule (min F, then larger k, then smaller m) rather than the listing's first-strictly-smaller
-//     scan, because the analysis relies on "ties -> larger batch".
+// O5. The exact dynamic programme of Section 5.1 (Algorithm 2), written as its recurrence.  With the
+//     requests of `ids` numbered 1..m, size_a = s_a + o_a, let D_a[k][c] be the smallest sum of o
+//     over the k-subsets of requests 1..a whose sizes add up to exactly c (infinite if there is
+//     none).  Then D_0[0][0] = 0 and
+//         D_a[k][c] = min( D_{a-1}[k][c],  D_{a-1}[k-1][c - size_a] + o_a ),
+//     where request a is recorded as taken in cell (a, k, c) only when the second term is strictly
+//     smaller (a tie keeps the subset without a; this is the listing's strict '<').  The batch is
+//     the cell of D_m with k >= 1, c <= M that minimises (F = D/k^2, then larger k, then smaller c)
+//     -- Section 3's tie rule, which the analysis relies on, instead of the listing's first-strictly-
+//     smaller scan -- and its members are read off by walking the taken marks back from a = m.
 // ---------------------------------------------------------------------------------------------
 int orc_phase1_dp(int m, const int* ids, const int* s, const int* o, i64 M,
                   int* chosen, i64* sum_o_out, i64* mem_out) {
     if (m > 128 || M > (1 << 22)) return -1;
     const i64 INF = INT64_MAX;
-    const int W = (int)M + 1;
-    std::vector<i64> dp((size_t)(m + 1) * W, INF);
-    struct Bits { uint64_t w[2]; };
-    std::vector<Bits> path((size_t)(m + 1) * W, Bits{{0, 0}});
-    dp[0] = 0;
-    for (int a = 0; a < m; ++a) {
-        int mi = s[ids[a]] + o[ids[a]], oi = o[ids[a]];
-        for (int k = a; k >= 0; --k)                    // k <= a: at most a requests seen so far
-            for (int mm = 0; mm + mi <= M; ++mm) {
-                i64 cur = dp[(size_t)k * W + mm];
-                if (cur == INF) continue;
-                i64 nv = cur + oi;
-                size_t dst = (size_t)(k + 1) * W + mm + mi;
-                if (nv < dp[dst]) {
-                    dp[dst] = nv;
-                    path[dst] = path[(size_t)k * W + mm];
-                    path[dst].w[a >> 6] |= 1ull << (a & 63);
-                }
+    const size_t W = (size_t)M + 1, layer = (size_t)(m + 1) * W;
+    std::vector<i64> prev(layer, INF), cur(layer, INF);
+    std::vector<std::vector<bool>> taken(m, std::vector<bool>(layer, false));
+    prev[0] = 0;
+    for (int a = 1; a <= m; ++a) {
+        const i64 size_a = (i64)s[ids[a - 1]] + o[ids[a - 1]], o_a = o[ids[a - 1]];
+        for (int k = 0; k <= a; ++k)                 // a subset of requests 1..a has at most a members
+            for (i64 c = 0; c <= M; ++c) {
+                i64 without = prev[k * W + c], with = INF;
+                if (k >= 1 && c >= size_a && prev[(k - 1) * W + (c - size_a)] != INF)
+                    with = prev[(k - 1) * W + (c - size_a)] + o_a;
+                const bool take = with < without;
+                cur[k * W + c] = take ? with : without;
+                taken[a - 1][k * W + c] = take;
             }
+        prev.swap(cur);
     }
-    int bestK = 0; i64 bestSum = 0; int bestM = 0;
+    int bestK = 0; i64 bestSum = 0, bestC = 0;
     for (int k = 1; k <= m; ++k)
-        for (int mm = 0; mm <= M; ++mm) {
-            i64 v = dp[(size_t)k * W + mm];
+        for (i64 c = 0; c <= M; ++c) {
+            const i64 v = prev[k * W + c];
             if (v == INF) continue;
-            bool better = bestK == 0;
-            if (!better) {
-                int c = orc_f_compare(v, k, bestSum, bestK);
-                better = c < 0;                          // equal (F, k): the smaller m was seen first
-            }
-            if (better) { bestK = k; bestSum = v; bestM = mm; }
+            // equal (F, k) keeps the cell seen first, which has the smaller c
+            if (bestK == 0 || orc_f_compare(v, k, bestSum, bestK) < 0) { bestK = k; bestSum = v; bestC = c; }
         }
-    const Bits& b = path[(size_t)bestK * W + bestM];
-    int c = 0;
-    for (int a = 0; a < m; ++a) if (b.w[a >> 6] >> (a & 63) & 1) chosen[c++] = ids[a];
+    std::vector<int> members;
+    {
+        int k = bestK; i64 c = bestC;
+        for (int a = m; a >= 1; --a)
+            if (taken[a - 1][k * W + c]) { members.push_back(ids[a - 1]); c -= (i64)s[ids[a - 1]] + o[ids[a - 1]]; --k; }
+    }
+    int cnt = 0;
+    for (auto it = members.rbegin(); it != members.rend(); ++it) chosen[cnt++] = *it;
     if (sum_o_out) *sum_o_out = bestSum;
-    if (mem_out) *mem_out = bestM;
-    return c;
+    if (mem_out) *mem_out = bestC;
+    return cnt;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -312,7 +316,7 @@ int orc_sorted_f_exact(int n, const int* s, const int* o, i64 M, int solver,
 // ---------------------------------------------------------------------------------------------
 // O6. Prefix-F batch selection -- a scalable stand-in for Algorithm 1's argmin that the paper does
 //     not print: candidates are restricted to prefixes of the remaining requests in the order
-//     Algorithm 4 starts from (ascending s+o; ties by o, then index).  From offset a, with
+//     Algorithm 3 starts from (ascending s+o; ties by o, then index).  From offset a, with
 //     k_max the longest prefix whose sum(s+o) <= M, pick k minimising (F, -k) over 1..k_max,
 //     append that prefix sorted by (o, index), continue from a + k.
 // ---------------------------------------------------------------------------------------------
@@ -410,6 +414,35 @@ int orc_eval_moves(int n, const int* s, const int* o, i64 M, const int* base,
     return 0;
 }
 
+// The same evaluation for the CPU-baseline timing: candidates split into contiguous shares over
+// `threads` host threads, each share evaluated exactly as above; form 0 = O2' (per-round occupancy
+// array), form 1 = O2 (Algorithm 1 Phase 2 literally, completion-time set tests).  Nothing but the
+// loop over candidates is parallel.
+int orc_eval_moves_threads(int n, const int* s, const int* o, i64 M, const int* base,
+                           i64 count, const int* type, const int* mi, const int* mj, i64* tel_out,
+                           int threads, int form) {
+    if (threads < 1) threads = 1;
+    if ((i64)threads > count) threads = (int)std::max<i64>(count, 1);
+    std::vector<int> rc(threads, 0);
+    auto work = [&](int w) {
+        const i64 lo = count * w / threads, hi = count * (w + 1) / threads;
+        std::vector<int> cand(n);
+        std::vector<i64> p(n);
+        for (i64 c = lo; c < hi; ++c) {
+            orc_apply_move(n, base, type[c], mi[c], mj[c], cand.data());
+            const int r = form == 1 ? orc_list_schedule_alg1(n, s, o, M, cand.data(), p.data(), &tel_out[c], 0)
+                                    : orc_list_schedule_rounds(n, s, o, M, cand.data(), p.data(), &tel_out[c], 0);
+            if (r) { rc[w] = -1; return; }
+        }
+    };
+    std::vector<std::thread> pool;
+    for (int w = 1; w < threads; ++w) pool.emplace_back(work, w);
+    work(0);
+    for (auto& th : pool) th.join();
+    for (int r : rc) if (r) return -1;
+    return 0;
+}
+
 // ---------------------------------------------------------------------------------------------
 // O8. Order-level local search.  neighbourhood 0 = all swaps, 1 = all swaps then all inserts,
 //     2 = `samples` sampled moves per iteration.  Per iteration: best = min (TEL, code) over the
@@ -501,13 +534,15 @@ i64 orc_bruteforce_best_order(int n, const int* s, const int* o, i64 M, int* bes
 
 
 // ---------------------------------------------------------------------------------------------
-// O10. Algorithm 4 (Local Swap Search), as printed: one batch out of the request set `ids`.
-//      Sort by ascending s+o (ties: lower index); first-fit fill in that order; then repeat: walk
-//      r_out over X and r_in over the requests outside X, take the FIRST pair that keeps
-//      sum(s+o) <= M and lowers F (|X| is fixed, so F drops iff o_in < o_out), swap, start over;
-//      stop when no pair qualifies.  Orders the listing leaves open: X is walked in insertion order
-//      with a swapped-in request taking the place of the one it replaces; the outside requests are
-//      walked in the sorted order.
+// O10. Local Swap Search (Section 5.2, Algorithm 3): one batch X out of the request set `ids`.
+//      Start: the requests by ascending size s+o (ties: lower index), filled first-fit under
+//      sum(s+o) <= M.  A swap (r_out in X, r_in outside X) is IMPROVING when the batch still fits,
+//      sum(s+o) - size(r_out) + size(r_in) <= M, and F drops; |X| does not change under a swap, so F
+//      drops exactly when o_in < o_out.  The search applies the first improving swap it meets and
+//      starts over, until X has no improving swap (a local optimum in Section 5.2's sense).
+//      "First" needs an order, which the paper leaves open: pairs are taken with r_out running over
+//      X in insertion order (a swapped-in request inherits the place of the one it replaced) and,
+//      for each r_out, r_in running over the outside requests in the sorted order.
 // Writes X (in its walking order) and returns |X|.  swaps_out (nullable) counts accepted swaps.
 // ---------------------------------------------------------------------------------------------
 int orc_local_swap_batch(int m, const int* ids, const int* s, const int* o, i64 M, int* chosen, i64* swaps_out) {
@@ -517,44 +552,37 @@ int orc_local_swap_batch(int m, const int* ids, const int* s, const int* o, i64 
         if (ta != tb) return ta < tb;
         return a < b;
     });
-    std::vector<int> X;
-    std::vector<char> inX(m, 0);                     // by position in I
-    std::vector<int> posX;                           // position in I of every member of X
+    auto size_of = [&](int r) { return (i64)s[r] + o[r]; };
+    std::vector<int> X;                              // members, in walking order
+    std::vector<int> where;                          // position in I of every member
+    std::vector<char> inside(m, 0);                  // by position in I
     i64 mem = 0, swaps = 0;
-    for (int p = 0; p < m; ++p) {
-        int r = I[p];
-        if (mem + s[r] + o[r] <= M) { X.push_back(r); posX.push_back(p); inX[p] = 1; mem += s[r] + o[r]; }
-    }
+    for (int p = 0; p < m; ++p)
+        if (mem + size_of(I[p]) <= M) { X.push_back(I[p]); where.push_back(p); inside[p] = 1; mem += size_of(I[p]); }
     if (X.empty()) return -1;
-    bool improved = true;
-    while (improved) {
-        improved = false;
-        i64 sum_o = 0;
-        for (int r : X) sum_o += o[r];
-        for (size_t k = 0; k < X.size() && !improved; ++k) {
-            int rout = X[k];
-            for (int p = 0; p < m; ++p) {
-                if (inX[p]) continue;
-                int rin = I[p];
-                i64 dm = (i64)(s[rin] + o[rin]) - (s[rout] + o[rout]);
-                if (mem + dm > M) continue;
-                i64 d_o = (i64)o[rin] - o[rout];
-                // newF < currentF with the same |X|:  (sum_o + d_o) / k^2 < sum_o / k^2
-                if (sum_o + d_o < sum_o) {
-                    inX[posX[k]] = 0; inX[p] = 1; posX[k] = p; X[k] = rin;
-                    mem += dm; improved = true; ++swaps;
-                    break;
-                }
-            }
-        }
+    auto improving = [&](size_t k, int p) {
+        if (inside[p]) return false;
+        if (mem - size_of(X[k]) + size_of(I[p]) > M) return false;
+        return o[I[p]] < o[X[k]];
+    };
+    for (;;) {
+        size_t k_hit = X.size(); int p_hit = -1;
+        for (size_t k = 0; k < X.size() && p_hit < 0; ++k)
+            for (int p = 0; p < m; ++p)
+                if (improving(k, p)) { k_hit = k; p_hit = p; break; }
+        if (p_hit < 0) break;
+        mem += size_of(I[p_hit]) - size_of(X[k_hit]);
+        inside[where[k_hit]] = 0; inside[p_hit] = 1;
+        where[k_hit] = p_hit; X[k_hit] = I[p_hit];
+        ++swaps;
     }
     for (size_t k = 0; k < X.size(); ++k) chosen[k] = X[k];
     if (swaps_out) *swaps_out = swaps;
     return (int)X.size();
 }
 
-// Sorted-F with Algorithm 4 as the Phase-1 solver (what Section 7 calls Sorted-F with Local Swap
-// Search): repeat { X = Algorithm 4 on the remaining requests; sort X by (o, index); append }.
+// Sorted-F with Algorithm 3 as the Phase-1 solver (what Section 7 calls Sorted-F with Local Swap
+// Search): repeat { X = Algorithm 3 on the remaining requests; sort X by (o, index); append }.
 int orc_sorted_f_local_swap(int n, const int* s, const int* o, i64 M, int* order, int* batch_offsets, i64* swaps_out) {
     std::vector<int> rem(n);
     std::iota(rem.begin(), rem.end(), 0);
@@ -586,7 +614,7 @@ int orc_sorted_f_local_swap(int n, const int* s, const int* o, i64 M, int* order
 //      G(X) = sum (alpha * s_i + o_i) / |X|^2 with alpha = a_num / a_den >= 0; alpha = 0 is F.
 //      Compared exactly on the integer weights w_i = a_num * s_i + a_den * o_i (a common factor
 //      a_den does not change the order).  Everything else as in O6 (prefix selection) and O10
-//      (Algorithm 4, where a swap now improves iff w_in < w_out).
+//      (Algorithm 3, where a swap now improves iff w_in < w_out).
 // ---------------------------------------------------------------------------------------------
 int orc_sorted_g_prefix(int n, const int* s, const int* o, i64 M, i64 a_num, i64 a_den, int* order, int* batch_offsets) {
     if (a_num < 0 || a_den <= 0) return -1;
@@ -660,7 +688,7 @@ int orc_sorted_g_local_swap(int n, const int* s, const int* o, i64 M, i64 a_num,
 
 
 // ---------------------------------------------------------------------------------------------
-// O12. Algorithm 5 (Quantile Greedy Selection): one batch out of the request set `ids`.
+// O12. Algorithm 4 (Quantile Greedy Selection): one batch out of the request set `ids`.
 //      I = ids sorted by ascending o (ties: lower index).  Q_p and Q_o are the 0.3-quantiles of
 //      s+o and of o over `sample`.  Pass 1 walks I and admits r when s_r+o_r <= Q_p, o_r <= Q_o
 //      and it still fits (mem + s_r + o_r <= M).  Pass 2 walks the requests left over, sorted by
@@ -703,7 +731,7 @@ int orc_quantile_greedy_batch(int m, const int* ids, const int* s, const int* o,
     return (int)X.size();
 }
 
-// The "random subset" of Algorithm 5, made reproducible: request id of batch number `batch` gets
+// The "random subset" of Algorithm 4, made reproducible: request id of batch number `batch` gets
 // the key mix(seed ^ mix(batch * 2^32 + id)) (splitmix64 finaliser); the sample is the
 // max(1, floor(m/2)) requests with the smallest keys, equal keys in the order of I (ascending o,
 // then index).  Writes the sample, returns its size.
@@ -722,7 +750,7 @@ int orc_quantile_sample(int m, const int* ids, const int* o, uint64_t seed, int 
     return size;
 }
 
-// Sorted-F with Algorithm 5 as the Phase-1 solver: repeat { sample; X = Algorithm 5 on the
+// Sorted-F with Algorithm 4 as the Phase-1 solver: repeat { sample; X = Algorithm 4 on the
 // remaining requests; sort X by (o, index); append }.
 int orc_sorted_f_quantile(int n, const int* s, const int* o, i64 M, uint64_t seed, int* order, int* batch_offsets) {
     std::vector<int> rem(n);
@@ -763,7 +791,7 @@ int orc_sorted_f_quantile(int n, const int* s, const int* o, i64 M, uint64_t see
 //                  the arrivals since the last recomputation reach half of the backlog size at that
 //                  recomputation.  Recomputation: sort the pending requests by ascending
 //                  (s+o, index); the first `lookahead` of them are ordered by Sorted-F with
-//                  Algorithm 4 (batch after batch, each batch by ascending (o, index)), the others
+//                  Algorithm 3 (batch after batch, each batch by ascending (o, index)), the others
 //                  follow in the (s+o, index) order.
 //      Left open by the text and fixed here: integer arrival times and "seen from iteration a+1";
 //      which pending requests form the look-ahead window (the first `lookahead` in the fallback
@@ -852,7 +880,7 @@ int orc_online_schedule(int n, const int* a, const int* s, const int* o, i64 M, 
 
 
 // ---------------------------------------------------------------------------------------------
-// O14. Sorted-F + A_min, Phase 2 (Section 5.5 "Handling Prediction Uncertainty", Algorithm 6):
+// O14. Sorted-F + A_min, Phase 2 (Section 5.5 "Handling Prediction Uncertainty", Algorithm 5):
 //      the executor when only a lower bound l_i <= o_i of every decode length is known.  Every
 //      request carries a running estimate e_i, initially l_i.  Iteration t = 1, 2, ...:
 //        1. requests that have run their o_i rounds leave; every other active request j is about

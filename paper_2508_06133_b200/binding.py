@@ -22,7 +22,7 @@ NBHD_SWAP, NBHD_SWAP_INSERT, NBHD_SAMPLED = 0, 1, 2
 EXPORTS = [
     "sched_init", "sched_init_batch", "sched_set_stream", "sched_sync", "sched_set_prefill_weight", "sched_set_base_order",
     "sched_get_base_order", "sched_eval_batch", "sched_eval_batch_dev", "sched_sweep_dev",
-    "sched_sorted_f", "sched_sorted_f_dev", "sched_sorted_f_local_swap", "sched_sorted_f_local_swap_dev", "sched_sorted_f_dp", "sched_sorted_f_quantile", "sched_online_simulate", "sched_amin_simulate", "sched_sorted_f_amin", "sched_local_search", "sched_accept_move", "sched_last_eval_kernel_ms", "sched_argmin_static_dev", "sched_release_cached_memory", "sched_stats", "sched_destroy",
+    "sched_sorted_f", "sched_sorted_f_dev", "sched_sorted_f_local_swap", "sched_sorted_f_local_swap_dev", "sched_sorted_f_dp", "sched_sorted_f_quantile", "sched_online_simulate", "sched_amin_simulate", "sched_sorted_f_amin", "sched_local_search", "sched_accept_move", "sched_last_eval_kernel_ms", "sched_argmin_static_dev", "sched_probe_peaks", "sched_debug_set_loop_cap", "sched_release_cached_memory", "sched_stats", "sched_destroy",
     "sched_strerror", "sched_last_cuda_error",
 ]
 
@@ -77,6 +77,8 @@ def load():
     lib.sched_stats.argtypes = [vp, vp, vp]
     lib.sched_last_eval_kernel_ms.argtypes = [vp, vp]
     lib.sched_argmin_static_dev.argtypes = [vp, i64, i64, vp, vp]
+    lib.sched_probe_peaks.argtypes = [vp, i32, i32, vp]
+    lib.sched_debug_set_loop_cap.argtypes = [i32]
     lib.sched_destroy.argtypes = [vp]
     lib.sched_strerror.argtypes = [C.c_int]
     lib.sched_strerror.restype = C.c_char_p
@@ -229,7 +231,7 @@ class Scheduler:
         return order, offs[:nb.value + 1].copy(), tel.value
 
     def sorted_f_local_swap(self):
-        """Sorted-F with Algorithm 4 as Phase-1 solver.  Returns (order, batch_offsets, TEL)."""
+        """Sorted-F with Algorithm 3 as Phase-1 solver.  Returns (order, batch_offsets, TEL)."""
         order = np.empty(self.n, dtype=np.int32)
         offs = np.zeros(self.n + 1, dtype=np.int32)
         nb, tel = C.c_int32(0), C.c_int64(0)
@@ -248,7 +250,7 @@ class Scheduler:
         return order, offs[:nb.value + 1].copy(), tel.value
 
     def sorted_f_quantile(self, seed=0):
-        """Sorted-F with Quantile Greedy Selection (Algorithm 5) as Phase-1 solver.
+        """Sorted-F with Quantile Greedy Selection (Algorithm 4) as Phase-1 solver.
         Returns (order, batch_offsets, TEL)."""
         order = np.empty(self.n, dtype=np.int32)
         offs = np.zeros(self.n + 1, dtype=np.int32)
@@ -287,6 +289,25 @@ class Scheduler:
 def release_cached_memory():
     """Return the library's cached device blocks to the driver (sched_release_cached_memory)."""
     _check(load().sched_release_cached_memory(), "sched_release_cached_memory")
+
+
+def debug_set_loop_cap(cap):
+    """Lower (cap >= 0) or restore (cap < 0) the iteration caps of the library's device loops on the
+    current device -- test support, see sched_debug_set_loop_cap."""
+    _check(load().sched_debug_set_loop_cap(int(cap)), "sched_debug_set_loop_cap")
+
+
+PROBE_NAMES = ("int_add", "int_add_max", "int_mad", "sim_mix", "smem_load", "smem_store", "int_alu")
+
+
+def probe_peaks(repeats=5, stream=None):
+    """Peak rates of the current CUDA device from the library's probe kernels (sched_probe_peaks):
+    dict name -> lane operations per second (the four integer probes) or bytes per second (shared
+    memory), measured now, at the clock the device runs at."""
+    out = np.zeros(len(PROBE_NAMES), dtype=np.float64)
+    ptr = C.c_void_p(stream.cuda_stream) if stream is not None else None
+    _check(load().sched_probe_peaks(_np_ptr(out), len(out), int(repeats), ptr), "sched_probe_peaks")
+    return dict(zip(PROBE_NAMES, out.tolist()))
 
 
 def argmin_static_dev(tel, best_out, *, count=None, index_base=0, stream=None):
@@ -343,7 +364,7 @@ def amin_simulate(n_each, s, lower, o, M, order):
 
 
 def sorted_f_amin(s, lower, o, M, phase1=0):
-    """Sorted-F + A_min for one backlog: Phase 1 on the lower bounds (0: prefix-F, 1: Algorithm 4), then
+    """Sorted-F + A_min for one backlog: Phase 1 on the lower bounds (0: prefix-F, 1: Algorithm 3), then
     the adaptive executor.  Returns (order, start times, TEL, evictions, peak memory)."""
     s = np.ascontiguousarray(s, dtype=np.int32)
     lower = np.ascontiguousarray(lower, dtype=np.int32)

@@ -11,6 +11,9 @@ NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", 
               "-shared", "-Xcompiler", "-fPIC", "-cudart", "shared"]
 
 
+UNITS = ["api.cu", "argmin_static.cu", "probe.cu"]          # translation units; the .cuh files are included by api.cu
+
+
 def sources():
     return sorted(os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".cu", ".cuh"))) + \
         [os.path.join(os.path.dirname(_HERE), "include", "kvsched.h")]
@@ -27,7 +30,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if force or stale():
         nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
         tmp = LIB + ".%d.tmp" % os.getpid()
-        cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + [os.path.join(CSRC, "api.cu"), os.path.join(CSRC, "argmin_static.cu"), "-o", tmp]
+        cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + [os.path.join(CSRC, f) for f in UNITS] + ["-o", tmp]
         subprocess.check_call(cmd)
         os.replace(tmp, LIB)
     return LIB

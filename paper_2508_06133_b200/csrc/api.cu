@@ -545,9 +545,12 @@ int sched_eval_batch_dev(sched_handle h, int kind, int64_t count, const void* ca
 #define RUN(N) k3_eval_policy<N><<<(unsigned)ctas, 32, smem, h->stream>>>(h->d_s, h->d_o, n, h->L, (int)h->M, \
                                                                   (const int*)candidates, (int)count,        \
                                                                   (i64*)tel_out, starts_out, h->d_status)
+        KV_CUDA(cudaEventRecord(h->ev_k3_begin, h->stream));
         KV_DISPATCH_SIM(h, RUN);
 #undef RUN
         KV_TRY(check_launch(h));
+        KV_CUDA(cudaEventRecord(h->ev_k3_end, h->stream));
+        h->ev_valid = true;
         h->evaluations += ctas;
         if (feasible_out) KV_CUDA(cudaMemsetAsync(feasible_out, 1, (size_t)ctas, h->stream));
         return SCHED_OK;
@@ -678,6 +681,7 @@ int sched_sweep_dev(sched_handle h, int sampled, uint64_t seed, int32_t iteratio
     KV_ENTER(h);
     if (h->batch_handle || h->n < 2 || count <= 0 || first_code < 0 || !best_out) return SCHED_E_INVAL;
     if (!sampled && first_code + count > neighbourhood_size(h->n, SCHED_NBHD_SWAP_INSERT, 0)) return SCHED_E_INVAL;
+    if (((uintptr_t)tel_out & 7) || ((uintptr_t)best_out & 7)) return SCHED_E_INVAL;
     i64* tel = (i64*)tel_out;
     for (i64 done = 0; done < count; done += kSweepChunk) {
         const i64 c = count - done < kSweepChunk ? count - done : kSweepChunk;
@@ -717,7 +721,7 @@ static int sorted_f_common_dev(sched_handle h, int solver, int32_t* order_out, i
     } else if (solver == 3) {
         KV_TRY(phase1_quantile(h, seed));
     } else {
-        // Algorithm 4: ascending (s+o, index), then first fit + improving swaps, batch after batch
+        // Algorithm 3: ascending (s+o, index), then first fit + improving swaps, batch after batch
         if (!h->d_ls) KV_TRY(dev_alloc(&h->d_ls, 7 * (size_t)n + 32));
         k1_keys_total_size<<<(n + 255) / 256, 256, 0, st>>>(h->d_s, h->d_o, n, h->d_keys_a, h->d_vals_a, SCHED_POLICY_TOTAL_SIZE);
         KV_TRY(check_launch(h));
@@ -830,7 +834,7 @@ static int phase1_dp(sched_handle h) {
     return rc;
 }
 
-// Algorithm 5 batch after batch; leaves the batches (members in ascending (o, index)) in d_vals_a and
+// Algorithm 4 batch after batch; leaves the batches (members in ascending (o, index)) in d_vals_a and
 // the boundaries in d_batch_off / d_num_batches.  Reads the batch size back once per batch.
 static int phase1_quantile(sched_handle h, u64 seed) {
     const int n = h->n;
@@ -1218,6 +1222,14 @@ int sched_sorted_f_amin(int32_t n, const int32_t* s, const int32_t* lower, const
         rc = amin_run(1, n, &n, s, lower, o, M, nullptr, h->d_order, start_out, tel_out, evictions_out, peak_out, nullptr);
     sched_destroy(h);
     return rc;
+}
+
+int sched_debug_set_loop_cap(int32_t cap) {
+    const int v = cap < 0 ? 0x7fffffff : cap;
+    KV_CUDA(cudaDeviceSynchronize());           // no kernel of this device may see the value change under it
+    KV_CUDA(cudaMemcpyToSymbol(kv_test_loop_cap, &v, sizeof(int)));
+    KV_CUDA(cudaDeviceSynchronize());
+    return SCHED_OK;
 }
 
 int sched_release_cached_memory(void) {

@@ -106,6 +106,14 @@ __device__ __forceinline__ int kv_lane() { return threadIdx.x & 31; }
 __device__ __forceinline__ int kv_warp_max(int v) { return __reduce_max_sync(KV_FULL, v); }
 __device__ __forceinline__ int kv_warp_min(int v) { return __reduce_min_sync(KV_FULL, v); }
 
+// Every device loop whose trip count depends on data carries a cap (its natural bound by
+// construction); a loop that reaches it records KV_DEV_LOOP_CAP in the status word and leaves, and
+// the host call returns SCHED_E_INTERNAL.  kv_test_loop_cap lowers every cap at once so that a test
+// can watch that path work (sched_debug_set_loop_cap); INT_MAX leaves the natural bounds alone.
+__constant__ int kv_test_loop_cap = 0x7fffffff;
+__device__ __forceinline__ int kv_loop_cap(int natural) { return min(natural, kv_test_loop_cap); }
+__device__ __forceinline__ i64 kv_loop_cap(i64 natural) { return natural < (i64)kv_test_loop_cap ? natural : (i64)kv_test_loop_cap; }
+
 // splitmix64 step, used by the sampled neighbourhood (published generator by Steele, Lea, Flood).
 __host__ __device__ __forceinline__ u64 kv_mix64(u64 z) {
     z += 0x9E3779B97F4A7C15ull;
@@ -118,10 +126,15 @@ struct Move { int type, i, j; };     // type 0 = swap (i < j), 1 = insert i -> j
 
 // Move code -> (type, i, j).  Swaps are numbered row by row: row i holds n-1-i codes and starts at
 // i*(2n-i-1)/2.  The row is first guessed from a square root and then corrected with exact integer
-// comparisons, so the result does not depend on floating-point rounding.
+// comparisons, so the result does not depend on floating-point rounding.  A code outside
+// 0 .. n(n-1)/2 + n(n-1) - 1 (compared in 64 bits, before any narrowing) decodes to {-1, -1, -1}.
 __host__ __device__ __forceinline__ Move kv_decode_move(int n, i64 code) {
     Move m;
     i64 nsw = (i64)n * (n - 1) / 2;
+    if (code < 0 || code >= 3 * nsw) {              // outside the neighbourhood: no move (callers reject i, j < 0)
+        m.type = -1; m.i = -1; m.j = -1;
+        return m;
+    }
     if (code < nsw) {
         double b = 2.0 * n - 1.0;
         i64 i = (i64)((b - sqrt(b * b - 8.0 * (double)code)) * 0.5);

@@ -2,7 +2,7 @@
 // (CTAs stride over the segments when there are more segments than CTAs).
 //
 // Used for the request orderings the method needs: ascending (s+o, o, index) over the whole
-// backlog (the order Algorithm 4 starts from), ascending (o, index) inside every selected batch
+// backlog (the order Algorithm 3 starts from), ascending (o, index) inside every selected batch
 // (Algorithm 1, Phase 1: "sort requests in X* in nondecreasing order of o_i"), and the order
 // policies.  Keys are built so that they are unique (the request index is part of the key or the
 // input is in index order), hence the result does not depend on anything but the keys.

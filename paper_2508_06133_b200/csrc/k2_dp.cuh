@@ -1,4 +1,4 @@
-// K2c -- Algorithm 2 (exact dynamic programme, Section 5.1 / Appendix D) as the Phase-1 solver.
+// K2c -- Algorithm 2 (exact dynamic programme, Section 5.1 / the supplement to Section 5) as the Phase-1 solver.
 //
 //   dp[k][m] = min { sum of o over X : |X| = k, sum of (s+o) over X = m },   m <= M,
 // built by taking the remaining requests one at a time (ascending index); a cell is overwritten only

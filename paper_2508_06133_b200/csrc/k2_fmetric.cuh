@@ -2,8 +2,8 @@
 //
 // Section 3: F(X) = (sum of o over X) / |X|^2; the batch with the smallest F is taken next, ties go
 // to the larger batch.  Candidates here are the prefixes of the not-yet-selected requests in
-// ascending (s+o, o, index) order (the order Algorithm 4 builds its first batch from), subject to
-// Algorithms 2/4/5's memory test  sum (s_i + o_i) <= M.  With inclusive prefix sums P (of s+o) and
+// ascending (s+o, o, index) order (the order Algorithm 3 builds its first batch from), subject to
+// Algorithms 2/3/4's memory test  sum (s_i + o_i) <= M.  With inclusive prefix sums P (of s+o) and
 // O (of o) over the sorted list, the batch that starts at offset a is
 //     k_max = max { k : P[a+k] - P[a] <= M },    k* = argmin_{1 <= k <= k_max} (O[a+k] - O[a]) / k^2,
 // and the next batch starts at a + k*.  F values are compared exactly: A/ka^2 < B/kb^2 iff

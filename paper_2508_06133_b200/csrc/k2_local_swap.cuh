@@ -1,8 +1,8 @@
-// K2b -- Phase 1 of Sorted-F with Algorithm 4 (Local Swap Search, Section 5.2 / Appendix D) as the
+// K2b -- Phase 1 of Sorted-F with Algorithm 3 (Local Swap Search, Section 5.2 / the supplement to Section 5) as the
 // batch solver, all batches in one launch of one CTA (the batches depend on each other: each one
 // is built from what the previous ones left).
 //
-// Algorithm 4 on the remaining requests, sorted by ascending s+o (ties: lower index):
+// Algorithm 3 on the remaining requests, sorted by ascending s+o (ties: lower index):
 //   first fit  -- in that order a request is taken iff it still fits; because the sizes ascend,
 //                 the result is the longest prefix whose sum(s+o) <= M;
 //   improvement -- walk r_out over X (insertion order, a swapped-in request keeps the place of the
@@ -55,7 +55,7 @@ struct K2lShared {
     i64 mem;
 };
 
-// One batch of Algorithm 4 out of the entries of sorted_ids[0 .. n) (request ids by ascending
+// One batch of Algorithm 3 out of the entries of sorted_ids[0 .. n) (request ids by ascending
 // (s+o, index)) whose `removed` flag is clear.  Called by all K2L_THREADS threads of a CTA; the
 // scratch arrays hold n ints each and may live in shared or global memory.  Writes the batch in X's
 // walking order to out[0 .. k0), sets the members' removed flags and returns k0 (the same value
@@ -145,7 +145,7 @@ __device__ int k2l_batch(const int* s, const int* o, const int* sorted_ids, int 
         __syncthreads();
         if (sh.pick[0] == INT_MAX) break;
         mem = sh.mem;
-        if (step > step_cap) { if (tid == 0) atomicExch(status, KV_DEV_LOOP_CAP); break; }
+        if (step > kv_loop_cap(step_cap)) { if (tid == 0) atomicExch(status, KV_DEV_LOOP_CAP); break; }
         __syncthreads();
     }
     // (d) hand the batch out and retire its requests

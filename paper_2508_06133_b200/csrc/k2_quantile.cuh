@@ -1,4 +1,4 @@
-// K2d -- Algorithm 5 (Quantile Greedy Selection, Section 5.3) as the Phase-1 solver.
+// K2d -- Algorithm 4 (Quantile Greedy Selection, Section 5.3) as the Phase-1 solver.
 //
 // One batch out of the remaining requests, which are kept as a list `rem` in ascending (o, index)
 // -- the order the algorithm sorts by first; taking a batch out keeps the list sorted, so it is

@@ -24,15 +24,22 @@ k5_argmin(const i64* __restrict__ tel, i64 count, i64 index_base, const int* __r
     __shared__ bool is_last;
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
     i64 bv = INT64_MAX, bi = INT64_MAX;
-    const i64 pairs = count >> 1;
-    const longlong2* tel2 = reinterpret_cast<const longlong2*>(tel);      // cudaMalloc'd: 16-byte aligned
+    // the array may start on any 8-byte boundary: an odd first element is taken alone so that the
+    // 16-byte loads behind it are aligned
+    const int head = (count > 0 && ((unsigned long long)tel & 8ull)) ? 1 : 0;
+    const i64 pairs = (count - head) >> 1;
+    const longlong2* tel2 = reinterpret_cast<const longlong2*>(tel + head);
     for (i64 k = (i64)blockIdx.x * K5_THREADS + tid; k < pairs; k += (i64)gridDim.x * K5_THREADS) {
         const longlong2 v = tel2[k];
-        k5_take(bv, bi, v.x, index_base + (index_map ? (i64)index_map[2 * k] : 2 * k));
-        k5_take(bv, bi, v.y, index_base + (index_map ? (i64)index_map[2 * k + 1] : 2 * k + 1));
+        const i64 e = head + 2 * k;
+        k5_take(bv, bi, v.x, index_base + (index_map ? (i64)index_map[e] : e));
+        k5_take(bv, bi, v.y, index_base + (index_map ? (i64)index_map[e + 1] : e + 1));
     }
-    if ((count & 1) && blockIdx.x == 0 && tid == 0)
-        k5_take(bv, bi, tel[count - 1], index_base + (index_map ? (i64)index_map[count - 1] : count - 1));
+    if (blockIdx.x == 0 && tid == 0) {
+        if (head) k5_take(bv, bi, tel[0], index_base + (index_map ? (i64)index_map[0] : 0));
+        if ((count - head) & 1)
+            k5_take(bv, bi, tel[count - 1], index_base + (index_map ? (i64)index_map[count - 1] : count - 1));
+    }
     for (int d = 16; d >= 1; d >>= 1) {
         const i64 ov = __shfl_xor_sync(KV_FULL, bv, d), oi = __shfl_xor_sync(KV_FULL, bi, d);
         k5_take(bv, bi, ov, oi);
@@ -78,12 +85,13 @@ __global__ void k5_accept_move(int* __restrict__ order, int n, const i64* __rest
     __shared__ int sh_do;
     __shared__ Move mv;
     if (threadIdx.x == 0) {
-        const bool improve = best[1] != INT64_MAX && best[0] < *cur_tel;
-        sh_do = improve ? 1 : 0;
+        bool improve = best[1] != INT64_MAX && best[0] < *cur_tel;
         if (improve) {
             mv = sampled ? kv_sample_move(n, seed, iteration, best[1]) : kv_decode_move(n, best[1]);
-            *cur_tel = best[0];
+            if ((unsigned)mv.i >= (unsigned)n || (unsigned)mv.j >= (unsigned)n) improve = false;   // not a move of this list
         }
+        if (improve) *cur_tel = best[0];
+        sh_do = improve ? 1 : 0;
         *accepted = improve ? 1 : 0;
     }
     __syncthreads();

@@ -11,7 +11,7 @@
 //                   never been planned, `period` iterations after the last plan, when it had run
 //                   empty, or when the arrivals since the last plan reach half of the backlog at
 //                   that plan.  A plan sorts the pending requests by ascending (s+o, index), orders
-//                   the first `lookahead` of them by Sorted-F with Algorithm 4 (batch after batch,
+//                   the first `lookahead` of them by Sorted-F with Algorithm 3 (batch after batch,
 //                   every batch by ascending (o, index)) and lets the others follow in sorted order.
 //
 // The iterations are not walked one by one.  Nothing changes between two iterations unless a
@@ -116,7 +116,7 @@ __global__ void __launch_bounds__(K6_THREADS) k6_online(const OnlineParams P) {
     int* ring = so + P.n_max;
     int* C = ring + P.L;                 // Sorted-F-Online: the cached list; SOF: started flags
     int* C2 = C + P.n_max;
-    int* win = C2 + P.n_max;             // 9 arrays of `lookahead` ints for Algorithm 4
+    int* win = C2 + P.n_max;             // 9 arrays of `lookahead` ints for Algorithm 3
     int* removed = win + W;
     int* rem = removed + W;
     int* remT = rem + W;
@@ -149,7 +149,7 @@ __global__ void __launch_bounds__(K6_THREADS) k6_online(const OnlineParams P) {
     i64 latency = 0;
 
     for (i64 turn = 0; remaining > 0; ++turn) {
-        if (turn > turn_cap) { if (tid == 0) atomicExch(P.status, KV_DEV_LOOP_CAP); break; }
+        if (turn > kv_loop_cap(turn_cap)) { if (tid == 0) atomicExch(P.status, KV_DEV_LOOP_CAP); break; }
         // arrivals seen by iteration t
         const int old = nvis;
         while (nvis < n && sa[nvis] <= t - 1) ++nvis;

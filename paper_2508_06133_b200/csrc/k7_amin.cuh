@@ -1,5 +1,5 @@
 // K7 -- Sorted-F + A_min, Phase 2 (Section 5.5 "Handling Prediction Uncertainty via Adaptive Output
-// Length Refinement"; Algorithm 6, Appendix D): the executor when only a lower bound l_i <= o_i of
+// Length Refinement"; Algorithm 5, the supplement to Section 5): the executor when only a lower bound l_i <= o_i of
 // every decode length is known.  Many independent scenarios (a backlog, its list and one vector of
 // lower bounds each), one CTA per scenario.
 //

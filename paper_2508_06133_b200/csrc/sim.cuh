@@ -1,4 +1,4 @@
-// Warp-level schedule simulator: Phase 2 of Algorithm 1 (Appendix C) for one ordered list.
+// Warp-level schedule simulator: Phase 2 of Algorithm 1 (the supplement to Section 3) for one ordered list.
 //
 // One warp owns one candidate.  Its state is the per-round occupancy of the requests admitted so
 // far, kept for the rounds x >= t (x is 0-based: x = tau - 1 for the paper's round tau) in a ring
@@ -78,7 +78,7 @@ __device__ __forceinline__ int sim_search_beyond(int* __restrict__ ring, int L, 
         delta += nd;
         lo = hi;
         hi = o + delta;
-        if (guard > L) { if (lane == 0) atomicExch(status, KV_DEV_LOOP_CAP); break; }
+        if (guard > kv_loop_cap(L)) { if (lane == 0) atomicExch(status, KV_DEV_LOOP_CAP); break; }
     }
     return delta;
 }

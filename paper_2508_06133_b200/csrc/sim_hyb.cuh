@@ -98,8 +98,7 @@ struct HybSim {
 
     // ---- passes over a window that ends inside the registers (as in the register simulator)
     template <int KLO, int KHI>
-    __device__ __forceinline__ int pass_max(int rl, int ol) const {
-        int v = (rl >= 0 && ol > 0) ? R[0] : -1;
+    __device__ __forceinline__ int pass_max_from(int v, int ol) const {
         constexpr int KI = KLO < KHI ? KLO : KHI;
 #pragma unroll
         for (int c = 1; c + 1 < KI; c += 2) v = __vimax3_s32(v, R[c], R[c + 1]);
@@ -110,78 +109,81 @@ struct HybSim {
     }
     template <int KLO, int KHI>
     __device__ __forceinline__ void pass_add(int rl, int ol, int k0) {
-        if (rl >= 0 && ol > 0) R[0] = kv_add_fma_pipe(R[0], k0);
+        if (rl >= 0 && ol > 0) R[0] = R[0] + k0;
 #pragma unroll
         for (int c = 1; c < KHI; ++c)
-            if (c < KLO || 32 * c < ol) R[c] = kv_add_fma_pipe(R[c], k0 + 32 * c);
+            if (c < KLO || 32 * c < ol) R[c] = R[c] + (k0 + 32 * c);
     }
-    template <int KLO, int KHI>
-    __device__ __forceinline__ int pass_need(int rl, int ol, int kadm) const {
-        int need = (rl >= 0 && ol > 0) ? min(R[0] + kadm, rl + 1) : 0;
+    // wait bound of every chunk behind the first, registers and far ring (rare path, see admit)
+    __device__ __forceinline__ int need_behind(int ol, int kadm, int nfar) const {
+        int need = 0;
 #pragma unroll
-        for (int c = 1; c < KHI; ++c)
-            if (c < KLO || 32 * c < ol) need = max(need, __viaddmin_s32(R[c], kadm, rl + 1 + 32 * c));
+        for (int c = 1; c < NREG; ++c)
+            if (32 * c < ol) need = max(need, __viaddmin_s32(R[c], kadm, rl + 1 + 32 * c));
+        for (int k = 0; k < nfar; ++k)
+            if (32 * (NREG + k) < ol)
+                need = max(need, __viaddmin_s32(far[32 * slot_of(k)], kadm, rl + 1 + 32 * (NREG + k)));
         return need;
     }
 
-    // Admit one request; returns its start.  All 32 lanes call this with identical (s, o).
+    // Admit one request; returns its start.  All 32 lanes call this with identical (s, o).  Same
+    // turn structure as the register simulator: the first chunk alone decides whether the request
+    // has to wait and for how long at least; otherwise the whole window is tested and, if it fits,
+    // the ramp is added; a window that reaches beyond the registers continues over the far ring.
     __device__ __forceinline__ int admit(int s, int o, int M, int lane, int* status) {
         int kadm = s + 1 - M - t;                      // V + kadm > 0  <=>  the cell is over budget
         for (int guard = 0;; ++guard) {
-            const int ol = o - rl, nch = (tm + o + 31) >> 5;
-            int delta = 0;
-            if (nch <= NREG) {
+            const int ol = o - rl;
+            const int v0 = (rl >= 0 && ol > 0) ? R[0] : -1;
+            int delta = kv_warp_max(__viaddmin_s32(v0, kadm, rl + 1));
+            if (delta <= 0) {
+                const int nch = (tm + o + 31) >> 5;
+                if (nch <= NREG) {
 #define KV_HS_TRY(A, B)                                                            \
-                {                                                                  \
-                    int vmax = pass_max<A, (B < NREG ? B : NREG)>(rl, ol);         \
-                    vmax = kv_warp_max(vmax);                                      \
-                    if (vmax + kadm <= 0) {                                        \
-                        pass_add<A, (B < NREG ? B : NREG)>(rl, ol, s + 1 + rl);    \
-                        tel += t + o;                                              \
-                        return t;                                                  \
-                    }                                                              \
-                    delta = pass_need<A, (B < NREG ? B : NREG)>(rl, ol, kadm);     \
-                }
-                KV_RS_BUCKETS(nch, KV_HS_TRY)
-#undef KV_HS_TRY
-            } else {
-                // every register is inside the window (R[0] from this lane's offset on), then the
-                // first nfar far chunks; far chunk k holds window offsets rl + 32 (NREG + k)
-                const int nfar = nch - NREG;
-                int v = rl >= 0 ? R[0] : -1;
-#pragma unroll
-                for (int c = 1; c + 1 < NREG; c += 2) v = __vimax3_s32(v, R[c], R[c + 1]);
-                for (int k = 0; k < nfar; ++k) {
-                    const int x = far[32 * slot_of(k)];
-                    v = max(v, (32 * (NREG + k) < ol) ? x : -1);
-                }
-                const int vmax = kv_warp_max(v);
-                if (vmax + kadm <= 0) {
-                    const int k0 = s + 1 + rl;
-                    if (rl >= 0) R[0] = kv_add_fma_pipe(R[0], k0);
-#pragma unroll
-                    for (int c = 1; c < NREG; ++c) R[c] = kv_add_fma_pipe(R[c], k0 + 32 * c);
-                    for (int k = 0; k < nfar; ++k) {
-                        if (32 * (NREG + k) < ol) {
-                            int* cell = far + 32 * slot_of(k);
-                            *cell += k0 + 32 * (NREG + k);
-                        }
+                    if constexpr ((A) < NREG) {                                    \
+                        int vmax = pass_max_from<A, (B < NREG ? B : NREG)>(v0, ol); \
+                        vmax = kv_warp_max(vmax);                                  \
+                        if (vmax + kadm <= 0) {                                    \
+                            pass_add<A, (B < NREG ? B : NREG)>(rl, ol, s + 1 + rl); \
+                            tel += t + o;                                          \
+                            return t;                                              \
+                        }                                                          \
                     }
-                    tel += t + o;
-                    return t;
-                }
-                int need = rl >= 0 ? min(R[0] + kadm, rl + 1) : 0;
+                    KV_RS_BUCKETS_MIX(nch, KV_HS_TRY)
+#undef KV_HS_TRY
+                    delta = kv_warp_max(need_behind(ol, kadm, 0));
+                } else {
+                    // every register is inside the window (R[0] from this lane's offset on), then the
+                    // first nfar far chunks; far chunk k holds window offsets rl + 32 (NREG + k)
+                    const int nfar = nch - NREG;
+                    int v = v0;
 #pragma unroll
-                for (int c = 1; c < NREG; ++c) need = max(need, __viaddmin_s32(R[c], kadm, rl + 1 + 32 * c));
-                for (int k = 0; k < nfar; ++k)
-                    if (32 * (NREG + k) < ol)
-                        need = max(need, __viaddmin_s32(far[32 * slot_of(k)], kadm, rl + 1 + 32 * (NREG + k)));
-                delta = need;
+                    for (int c = 1; c + 1 < NREG; c += 2) v = __vimax3_s32(v, R[c], R[c + 1]);
+                    for (int k = 0; k < nfar; ++k) {
+                        const int x = far[32 * slot_of(k)];
+                        v = max(v, (32 * (NREG + k) < ol) ? x : -1);
+                    }
+                    const int vmax = kv_warp_max(v);
+                    if (vmax + kadm <= 0) {
+                        const int k0 = s + 1 + rl;
+                        if (rl >= 0) R[0] = R[0] + k0;
+#pragma unroll
+                        for (int c = 1; c < NREG; ++c) R[c] = R[c] + (k0 + 32 * c);
+                        for (int k = 0; k < nfar; ++k) {
+                            if (32 * (NREG + k) < ol) {
+                                int* cell = far + 32 * slot_of(k);
+                                *cell += k0 + 32 * (NREG + k);
+                            }
+                        }
+                        tel += t + o;
+                        return t;
+                    }
+                    delta = kv_warp_max(need_behind(ol, kadm, nfar));
+                }
             }
-            delta = kv_warp_max(delta);                // >= 1: the worst cell alone asks for it
-            kadm -= delta;
+            kadm -= delta;                             // >= 1: the worst cell alone asks for it
             advance(delta, lane);
-            if (guard > span) { if (lane == 0) atomicExch(status, KV_DEV_LOOP_CAP); return t; }
+            if (guard > kv_loop_cap(span)) { if (lane == 0) atomicExch(status, KV_DEV_LOOP_CAP); return t; }
         }
     }
 };

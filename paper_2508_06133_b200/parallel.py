@@ -85,6 +85,19 @@ class SingleRank:
         return value
 
 
+def sharded_iteration(evaluator, comm, total, sampled, seed, iteration):
+    """One iteration of the search over ``total`` move indices: this rank sweeps its share, the ranks
+    agree on the smallest (TEL, index) pair -- all-reduce(min) of the TEL, then of the lowest index
+    among the ranks that attain it -- and every rank applies that pair through ``evaluator.accept``.
+    Returns (accepted, TEL of the base order afterwards, winning index, winning TEL)."""
+    first, count = shard(total, comm.rank, comm.world)
+    tel, idx = evaluator.sweep(first, count, sampled, seed, iteration) if count > 0 else (I64_MAX, I64_MAX)
+    best_tel = comm.min(tel)
+    best_idx = comm.min(idx if tel == best_tel else I64_MAX)
+    accepted, cur = evaluator.accept(best_tel, best_idx, sampled, seed, iteration)
+    return accepted, cur, best_idx, best_tel
+
+
 def sharded_local_search(evaluator, neighbourhood, iters, *, seed=0, samples_per_iter=0, comm=None):
     """Runs the search described in the module docstring.  ``evaluator`` has ``n``, ``base_tel()``,
     ``sweep(first, count, sampled, seed, iteration) -> (TEL, index)`` and
@@ -95,16 +108,11 @@ def sharded_local_search(evaluator, neighbourhood, iters, *, seed=0, samples_per
     comm = comm if comm is not None else SingleRank()
     sampled = neighbourhood == kv.NBHD_SAMPLED
     total = neighbourhood_size(evaluator.n, neighbourhood, samples_per_iter)
-    first, count = shard(total, comm.rank, comm.world)
     cur = evaluator.base_tel()
     trace = []
     done = 0
     while done < iters and total > 0:
-        it = done
-        tel, idx = evaluator.sweep(first, count, sampled, seed, it) if count > 0 else (I64_MAX, I64_MAX)
-        best_tel = comm.min(tel)
-        best_idx = comm.min(idx if tel == best_tel else I64_MAX)
-        accepted, cur = evaluator.accept(best_tel, best_idx, sampled, seed, it)
+        accepted, cur, best_idx, best_tel = sharded_iteration(evaluator, comm, total, sampled, seed, done)
         trace.append((best_idx, best_tel))
         done += 1
         if not accepted and not sampled:

@@ -66,7 +66,7 @@ def test_null_arguments(lib):
 
 
 def test_sources_name_no_closed_calls():
-    banned = ["cudaMemcpy" + "BatchAsync", "cudaMemcpy3D" + "BatchAsync", "multicast::cluster"]
+    banned = ["cudaMemcpy" + "BatchAsync", "cudaMemcpy3D" + "BatchAsync", "multicast" + "::cluster"]
     for dirpath, _, files in os.walk(os.path.join(ROOT, "paper_2508_06133_b200")):
         for f in files:
             if f.endswith((".cu", ".cuh", ".py", ".h")):

@@ -1,0 +1,105 @@
+"""GPU parity at the stated sizes of the two large configurations.
+
+* n = 10,000 (the headline backlog): ONE complete swap + insert sweep of the Sorted-F order, all
+  149,985,000 neighbours, through ``sched_sweep_dev`` with every TEL dumped.  The arg-min is
+  re-derived on the host from the dumped array, 10,000 uniformly drawn neighbours and the winning
+  one are re-evaluated by the CPU oracle, and the first iteration of ``sched_local_search`` over the
+  same neighbourhood must report the same (move, TEL) pair (Algorithm 1 Phase 2 scores every
+  neighbour; the improving rule of Section 5.2 decides on acceptance).
+* n = 100,000 (heavy tail, decode lengths up to 4,096): Sorted-F, then local-search iterations over
+  2^20 sampled moves each.  Every iteration's reported (sample index, TEL) is replayed through the
+  oracle's executor, and the final order must be the replay's.  Three iterations by default; the
+  configuration's 50 with ``KVSCHED_FULL_CONFIGS=1`` (about a quarter of an hour of GPU time).
+
+Both tests print one line with the wall time and the TELs (``pytest -s`` shows it).
+"""
+import os
+import time
+
+import numpy as np
+import pytest
+
+import oracle as orc
+from paper_2508_06133_b200 import binding as kv
+from paper_2508_06133_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+def test_mixed_10k_one_complete_swap_insert_sweep():
+    import torch
+    inst = W.mixed_10k()
+    n = inst.n
+    nsw = n * (n - 1) // 2
+    total = nsw + n * (n - 1)
+    assert total == 149_985_000
+    dev = torch.device("cuda", torch.cuda.current_device())
+    tel = torch.empty(total, dtype=torch.int64, device=dev)
+    best = torch.zeros(2, dtype=torch.int64, device=dev)
+    r_order, _ = orc.sorted_f_prefix(inst.s, inst.o, inst.M)
+    r_tel0 = orc.list_schedule_rounds(inst.s, inst.o, inst.M, r_order)[1]
+    with kv.Scheduler(inst.s, inst.o, inst.M) as h:
+        order, _, tel0 = h.sorted_f()
+        assert (order == r_order).all() and tel0 == r_tel0
+        t0 = time.perf_counter()
+        h.sweep_dev(total, best, first_code=0, tel_out=tel)
+        h.sync()
+        sweep_s = time.perf_counter() - t0
+        tels = tel.cpu().numpy()
+        del tel
+        # arg-min re-derived on the host: the first minimum is the lowest code among equal TELs
+        k = int(np.argmin(tels))
+        assert best.cpu().tolist() == [int(tels[k]), k]
+        # properties that hold for every neighbour
+        assert tels.min() >= int(inst.o.sum())
+        assert tels.max() < np.iinfo(np.int64).max
+        # 10,000 uniformly drawn codes, the extreme codes of both move types, and the winner
+        picks = (W.u64(2024, 3, np.arange(10_000)) % np.uint64(total)).astype(np.int64)
+        picks = np.concatenate([picks, [0, nsw - 1, nsw, total - 1, k]])
+        mv = [orc.decode_move(n, int(c)) for c in picks]
+        ref = orc.eval_moves(inst.s, inst.o, inst.M, r_order, [m[0] for m in mv], [m[1] for m in mv], [m[2] for m in mv])
+        assert (tels[picks] == ref).all()
+        best_tel = int(tels[k])
+        del tels
+        # the library's own search: its first iteration sweeps the same neighbourhood
+        t0 = time.perf_counter()
+        final, ftel, done, trace = h.local_search(kv.NBHD_SWAP_INSERT, 1)
+        search_s = time.perf_counter() - t0
+    assert done == 1 and trace.tolist() == [[k, best_tel]]
+    if best_tel < tel0:
+        moved = orc.apply_move(r_order, *orc.decode_move(n, k))
+        assert (final == moved).all() and ftel == best_tel
+        assert orc.list_schedule_rounds(inst.s, inst.o, inst.M, moved)[1] == best_tel
+    else:
+        assert (final == r_order).all() and ftel == tel0
+    print("\nmixed_10k complete sweep: %d neighbours in %.1f s (%.3e evals/s), search iteration %.1f s, "
+          "Sorted-F TEL %d -> best neighbour %d (code %d)" % (total, sweep_s, total / sweep_s, search_s, tel0, best_tel, k))
+
+
+def test_heavy_100k_sampled_local_search():
+    inst = W.heavy_100k()
+    n = inst.n
+    iters = 50 if os.environ.get("KVSCHED_FULL_CONFIGS") == "1" else 3
+    samples, seed = 1 << 20, 17
+    r_order, r_offs = orc.sorted_f_prefix(inst.s, inst.o, inst.M)
+    r_tel = orc.list_schedule_rounds(inst.s, inst.o, inst.M, r_order)[1]
+    with kv.Scheduler(inst.s, inst.o, inst.M) as h:
+        order, offs, tel0 = h.sorted_f()
+        assert (order == r_order).all() and (offs == r_offs).all() and tel0 == r_tel
+        t0 = time.perf_counter()
+        final, ftel, done, trace = h.local_search(kv.NBHD_SAMPLED, iters, seed=seed, samples_per_iter=samples)
+        wall = time.perf_counter() - t0
+    assert done == iters and len(trace) == iters
+    cur, cur_tel, accepted = r_order, r_tel, 0
+    for it, (m, best) in enumerate(trace):
+        assert 0 <= m < samples
+        cand = orc.apply_move(cur, *orc.sample_move(n, seed, it, int(m)))
+        assert orc.list_schedule_rounds(inst.s, inst.o, inst.M, cand)[1] == best
+        for mm in (0, samples // 2, samples - 1):                  # no sampled move beats the reported best
+            c2 = orc.apply_move(cur, *orc.sample_move(n, seed, it, mm))
+            assert orc.list_schedule_rounds(inst.s, inst.o, inst.M, c2)[1] >= best
+        if best < cur_tel:
+            cur, cur_tel, accepted = cand, int(best), accepted + 1
+    assert (final == cur).all() and ftel == cur_tel and ftel <= tel0
+    print("\nheavy_100k: %d iterations x %d sampled moves in %.1f s (%.3e evals/s), %d accepted, TEL %d -> %d"
+          % (iters, samples, wall, iters * samples / wall, accepted, tel0, ftel))

@@ -257,7 +257,7 @@ def test_sorted_f_example1(golden):
 
 
 def test_sorted_f_local_swap_matches_oracle():
-    """Sorted-F with Algorithm 4 (Local Swap Search) as Phase-1 solver: batches, order and TEL."""
+    """Sorted-F with Algorithm 3 (Local Swap Search) as Phase-1 solver: batches, order and TEL."""
     rng = np.random.default_rng(44)
     cases = [W.tiny(), W.mixed_1k(), W.paper_scale(), W.mixed_10k()]
     for trial in range(40):
@@ -307,7 +307,7 @@ def test_sorted_f_exact_dp_matches_oracle():
 
 
 def test_sorted_f_quantile_greedy_matches_oracle():
-    """Sorted-F with Algorithm 5 (Quantile Greedy Selection) as Phase-1 solver: batches, order, TEL."""
+    """Sorted-F with Algorithm 4 (Quantile Greedy Selection) as Phase-1 solver: batches, order, TEL."""
     rng = np.random.default_rng(46)
     cases = [W.tiny(), W.mixed_1k(), W.paper_scale(), W.mixed_10k()]
     for trial in range(60):
@@ -447,7 +447,7 @@ def _amin_rows(instances):
 
 
 def test_amin_small_scenarios_match_the_set_form_oracle():
-    """Algorithm 6's executor against the oracle that re-derives every projection from the sets:
+    """Algorithm 5's executor against the oracle that re-derives every projection from the sets:
     every final start time, TEL, eviction count and peak memory; tight and loose memories, exact,
     mild and crude lower bounds (l = 1 for everybody included), and the hand-worked cases."""
     rng = np.random.default_rng(71)
@@ -528,7 +528,7 @@ def test_amin_argument_errors():
 
 
 def test_tiny_backlog_all_solvers_and_brute_force():
-    """n = 16: prefix-F, Algorithm 4 and the exact DP orders, a full swap search from the DP order,
+    """n = 16: prefix-F, Algorithm 3 and the exact DP orders, a full swap search from the DP order,
     and all 8! orders of the first 8 requests against the oracle's brute force."""
     import itertools
     inst = W.tiny()
@@ -772,9 +772,11 @@ def test_device_pointer_candidates_are_bounds_checked_on_the_device():
     s, o = np.array([2, 3, 4, 5], dtype=np.int32), np.array([1, 2, 3, 1], dtype=np.int32)
     big = np.iinfo(np.int64).max
     with kv.Scheduler(s, o, 20) as h:
-        codes = torch.tensor([0, 17, 18, 10 ** 12, -5], dtype=torch.int64, device=dev)     # 6 swaps + 12 inserts: 0..17 valid
-        tel = torch.zeros(5, dtype=torch.int64, device=dev)
-        h.eval_batch_dev(kv.CAND_MOVE, 5, codes, tel)
+        # 6 swaps + 12 inserts: 0..17 valid; -1 sits next to code 0, and 18 + 2^33 * (n - 1) would wrap
+        # to row 0 of the inserts if the row were narrowed to 32 bits before the range check
+        codes = torch.tensor([0, 17, 18, 10 ** 12, -5, -1, 18 + (1 << 33) * 3], dtype=torch.int64, device=dev)
+        tel = torch.zeros(7, dtype=torch.int64, device=dev)
+        h.eval_batch_dev(kv.CAND_MOVE, 7, codes, tel)
         h.sync()
         got = tel.cpu().numpy()
         assert got[0] == oracle_moves(s, o, 20, np.arange(4), [0])[0] and got[1] == oracle_moves(s, o, 20, np.arange(4), [17])[0]
@@ -791,6 +793,38 @@ def test_device_pointer_candidates_are_bounds_checked_on_the_device():
         h.eval_batch_dev(kv.CAND_START_TIMES, 2, starts, tel, feas)
         h.sync()
         assert feas.cpu().numpy().tolist() == [int(orc.check_schedule(s, o, 20, [0, 0, 0, 0])["feasible"]), 0]
+
+
+def test_sweep_accepts_any_8_byte_aligned_tel_array():
+    """tel_out of a sweep may be a slice that starts on an odd element (8-byte but not 16-byte
+    aligned); a pointer that is not 8-byte aligned is refused on the host before any launch."""
+    import ctypes as C
+    import torch
+    dev = torch.device("cuda", torch.cuda.current_device())
+    inst = W.mixed_backlog(200, 21, 20000, name="offset")
+    n = inst.n
+    total = n * (n - 1) // 2 + n * (n - 1)
+    with kv.Scheduler(inst.s, inst.o, inst.M) as h:
+        h.sorted_f_dev()
+        ref_tel = torch.empty(total, dtype=torch.int64, device=dev)
+        ref_best = torch.zeros(2, dtype=torch.int64, device=dev)
+        h.sweep_dev(total, ref_best, tel_out=ref_tel)
+        for count in (total, total - 1, 1, 2):
+            buf = torch.full((total + 3,), -7, dtype=torch.int64, device=dev)
+            best = torch.zeros(2, dtype=torch.int64, device=dev)
+            h.sweep_dev(count, best, tel_out=buf[1:1 + count])
+            h.sync()
+            got = buf.cpu().numpy()
+            want = ref_tel[:count].cpu().numpy()
+            assert (got[1:1 + count] == want).all() and got[0] == -7 and (got[1 + count:] == -7).all()
+            k = int(np.argmin(want))
+            assert best.cpu().tolist() == [int(want[k]), k]
+        lib = kv.load()
+        buf = torch.zeros(16, dtype=torch.int64, device=dev)
+        best = torch.zeros(2, dtype=torch.int64, device=dev)
+        launches = h.stats()[0]
+        rc = lib.sched_sweep_dev(h._h, 0, 0, 0, 0, 4, C.c_void_p(buf.data_ptr() + 4), C.c_void_p(best.data_ptr()))
+        assert rc == kv.E_INVAL and h.stats()[0] == launches
 
 
 # ------------------------------------------------------------------------------------ errors on a live handle
@@ -819,6 +853,44 @@ def test_error_paths_on_a_handle():
         assert tel[0] == orc.list_schedule_alg1(s, o, 20, [2, 1, 0])[1]
         launches, evals = h.stats()
         assert launches > 0 and evals >= 1
+
+
+def test_a_loop_cap_that_runs_out_is_reported_and_leaves_the_handle_usable():
+    """With the device loops' caps lowered to zero iterations, the first request that has to wait makes
+    the simulator give up: the kernel ends normally, the call returns SCHED_E_INTERNAL, nothing
+    faults, and with the caps restored the same handle evaluates the same candidates correctly."""
+    inst = W.mixed_backlog(400, 31, 20000, name="cap")
+    orders = np.stack([np.arange(inst.n), np.arange(inst.n)[::-1]]).astype(np.int32)
+    ref = [orc.list_schedule_rounds(inst.s, inst.o, inst.M, r)[1] for r in orders]
+    with kv.Scheduler(inst.s, inst.o, inst.M) as h:
+        assert h.eval_batch(kv.CAND_ORDER, orders)[0].tolist() == ref
+        kv.debug_set_loop_cap(0)
+        try:
+            with pytest.raises(kv.SchedError) as e:
+                h.eval_batch(kv.CAND_ORDER, orders)
+            assert e.value.code == kv.E_INTERNAL
+            with pytest.raises(kv.SchedError) as e:
+                h.sorted_f()
+            assert e.value.code == kv.E_INTERNAL
+        finally:
+            kv.debug_set_loop_cap(-1)
+        assert h.eval_batch(kv.CAND_ORDER, orders)[0].tolist() == ref
+        order, _, tel = h.sorted_f()
+        r_order, _ = orc.sorted_f_prefix(inst.s, inst.o, inst.M)
+        assert (order == r_order).all() and tel == orc.list_schedule_rounds(inst.s, inst.o, inst.M, r_order)[1]
+    # the hybrid and the all-shared-memory simulators, and the policy kernel, report the same way
+    s2, o2, M2 = W.policy_sweep(num_instances=8)
+    pols = np.array([kv.POLICY_SORTED_F, kv.POLICY_FCFS], dtype=np.int32)
+    with kv.Scheduler.batch(s2, o2, M2) as h:
+        good = h.eval_batch(kv.CAND_POLICY, pols)[0]
+        kv.debug_set_loop_cap(0)
+        try:
+            with pytest.raises(kv.SchedError) as e:
+                h.eval_batch(kv.CAND_POLICY, pols)
+            assert e.value.code == kv.E_INTERNAL
+        finally:
+            kv.debug_set_loop_cap(-1)
+        assert (h.eval_batch(kv.CAND_POLICY, pols)[0] == good).all()
 
 
 # ------------------------------------------------------------------------------------ full-size configurations

@@ -1,6 +1,7 @@
-"""World-size-2 check (gloo, CPU) of how the benchmark spreads one sampled neighbourhood over ranks:
-disjoint contiguous sample slices, the same moves as a single rank would draw, and the
-max-over-ranks time reduction.  No GPU and no kernel is involved."""
+"""World-size-2 checks (gloo, CPU) of how the benchmark spreads one sampled neighbourhood over ranks
+(disjoint contiguous sample slices, the same moves as a single rank would draw, the max-over-ranks
+time reduction) and of the step it times under torchrun: one iteration of the sharded local search
+with its all-reduce(min) exchange.  No GPU and no kernel is involved."""
 import os
 import sys
 
@@ -20,13 +21,14 @@ def _worker(rank, world, port, out):
     dist.init_process_group("gloo", rank=rank, world_size=world)
     import bench
     count, n, seed, it = 1000, 500, 7, 3
-    first = bench.rank_first_sample(rank, count)
+    first, share = bench.rank_share(world * count, rank, world)
+    ok_share = share == count
     ty, mi, mj = bench.sampled_move_positions(n, seed, it, first, count)
     mine = torch.from_numpy(np.stack([ty, mi, mj]))
     gathered = [torch.zeros_like(mine) for _ in range(world)]
     dist.all_gather(gathered, mine)
     whole = np.stack(bench.sampled_move_positions(n, seed, it, 0, world * count))
-    ok = bool((torch.cat(gathered, dim=1).numpy() == whole).all())
+    ok = ok_share and bool((torch.cat(gathered, dim=1).numpy() == whole).all())
     firsts = [torch.zeros(1, dtype=torch.int64) for _ in range(world)]
     dist.all_gather(firsts, torch.tensor([first]))
     ok &= [int(f) for f in firsts] == [r * count for r in range(world)]
@@ -114,6 +116,18 @@ def _search_worker(rank, world, port, out):
         ok &= tel == r_tel and done == r_done and (trace == r_trace).all() and (ev.order == r_order).all()
         total = par.neighbourhood_size(n, nbhd, samples)
         ok &= all(fc == par.shard(total, rank, world) for fc in ev.sweeps) or total < world
+    # the step the benchmark times under torchrun: one iteration over a sampled neighbourhood split
+    # over the ranks, exchange included; both ranks must end with the oracle's pair and order
+    for samples, it in ((64, 0), (5, 1), (1, 2)):
+        ev = _OracleEvaluator(s, o, M, start)
+        accepted, cur, idx, tel = par.sharded_iteration(ev, par.TorchComm(device="cpu"), samples, True, 23, it)
+        mv = [orc.sample_move(n, 23, it, m) for m in range(samples)]
+        ref = orc.eval_moves(s, o, M, start, [m[0] for m in mv], [m[1] for m in mv], [m[2] for m in mv])
+        k = int(np.argmin(ref))
+        base_tel = orc.list_schedule_rounds(s, o, M, start)[1]
+        ok &= (idx, tel) == (k, int(ref[k])) and accepted == (int(ref[k]) < base_tel)
+        want = orc.apply_move(start, *mv[k]) if accepted else start
+        ok &= (ev.order == want).all() and cur == min(base_tel, int(ref[k]))
     # shares: contiguous, disjoint, complete, also when there are fewer indices than ranks
     for total in (0, 1, 2, 7, 1000, 149985000):
         parts = [par.shard(total, r, 8) for r in range(8)]

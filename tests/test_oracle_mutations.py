@@ -31,20 +31,20 @@ MUTATIONS = [
      "mem += s[r] + o[r];\n            if (mem >= M) break;\n            so += o[r];", "test_prefix_f_by_hand", False),
     ("insert code maps to the wrong target", "*type = 1; *i_out = i; *j_out = r < i ? r : r + 1;",
      "*type = 1; *i_out = i; *j_out = r <= i ? r : r + 1;", "test_move_codes_enumerate_the_neighbourhood", False),
-    ("Algorithm 4 memory test off by one", "if (mem + dm > M) continue;\n                i64 d_o",
-     "if (mem + dm >= M) continue;\n                i64 d_o", "test_local_swap_worked_by_hand", False),
+    ("Algorithm 3 memory test off by one", "if (mem - size_of(X[k]) + size_of(I[p]) > M) return false;",
+     "if (mem - size_of(X[k]) + size_of(I[p]) >= M) return false;", "test_local_swap_worked_by_hand", False),
     ("G-metric without the prefill term", "sw += a_num * s[r] + a_den * o[r];", "sw += a_den * o[r];",
      "test_sorted_g_reduces_to_f_and_differs_by_hand", False),
-    ("Algorithm 5 quantile position", "const int q = (int)((3ll * (sample_size - 1)) / 10);", "const int q = (int)((3ll * sample_size) / 10);",
+    ("Algorithm 4 quantile position", "const int q = (int)((3ll * (sample_size - 1)) / 10);", "const int q = (int)((3ll * sample_size) / 10);",
      "test_quantile_greedy_properties", False),
-    ("Algorithm 5 pass 2 stops at the first misfit", "for (int r : remaining) {\n        i64 T = (i64)s[r] + o[r];\n        if (mem + T <= M) { X.push_back(r); mem += T; }\n    }",
+    ("Algorithm 4 pass 2 stops at the first misfit", "for (int r : remaining) {\n        i64 T = (i64)s[r] + o[r];\n        if (mem + T <= M) { X.push_back(r); mem += T; }\n    }",
      "for (int r : remaining) {\n        i64 T = (i64)s[r] + o[r];\n        if (mem + T <= M) { X.push_back(r); mem += T; } else break;\n    }",
      "test_quantile_greedy_worked_by_hand", False),
-    ("Algorithm 5 ratio compared in floating point", "__int128 l = (__int128)o[a] * ((i64)s[b] + o[b]), r = (__int128)o[b] * ((i64)s[a] + o[a]);",
+    ("Algorithm 4 ratio compared in floating point", "__int128 l = (__int128)o[a] * ((i64)s[b] + o[b]), r = (__int128)o[b] * ((i64)s[a] + o[a]);",
      "double l = (double)o[a] / ((double)s[a] + o[a]), r = (double)o[b] / ((double)s[b] + o[b]);", "test_quantile_greedy_worked_by_hand", False),
-    ("Algorithm 5 without the output-length threshold", "if (T <= Qp && o[r] <= Qo && mem + T <= M)", "if (T <= Qp && mem + T <= M)",
+    ("Algorithm 4 without the output-length threshold", "if (T <= Qp && o[r] <= Qo && mem + T <= M)", "if (T <= Qp && mem + T <= M)",
      "test_quantile_greedy_worked_by_hand", False),
-    ("Algorithm 5 sample of the wrong size", "int size = m / 2 > 1 ? m / 2 : 1;", "int size = (m + 1) / 2;", "test_quantile_greedy_properties", False),
+    ("Algorithm 4 sample of the wrong size", "int size = m / 2 > 1 ? m / 2 : 1;", "int size = (m + 1) / 2;", "test_quantile_greedy_properties", False),
     ("online: early refresh at 100 % instead of 50 %", "|| 2 * new_since >= backlog_last) {", "|| new_since >= backlog_last) {",
      "test_sorted_f_online_worked_by_hand", False),
     ("online: a refused head is skipped", "if (!fits) break;\n            for (int j = 1; j <= o[r]; ++j) U[t - 1 + j] += (i64)s[r] + j;",
@@ -66,6 +66,10 @@ MUTATIONS = [
     ("per-round A_min grows an estimate without its memory", "else if (t - p[j] > est[j]) { est[j] = t - p[j]; proj[t % H] += s[j] + t - p[j]; }",
      "else if (t - p[j] > est[j]) { est[j] = t - p[j]; proj[t % H] += t - p[j]; }",
      "test_amin_per_round_form_equals_the_set_form", False),
+    ("Algorithm 1's batch constraint replaced by the sum test", "if (reading == 1) feas = mem <= M;", "if (reading == 1 || reading == 0) feas = mem <= M;",
+     "test_phase1_algorithm1_constraint_by_hand", False),
+    ("Algorithm 1's batch constraint counts requests that have already finished", "if ((mask >> b & 1) && o[ids[b]] >= o[ids[a]]) tot += (i64)s[ids[b]] + o[ids[a]];",
+     "if (mask >> b & 1) tot += (i64)s[ids[b]] + o[ids[a]];", "test_phase1_algorithm1_constraint_by_hand", False),
     ("shortest-output-first sorts by size", "std::stable_sort(order, order + n, [&](int a, int b) { return o[a] < o[b]; });",
      "std::stable_sort(order, order + n, [&](int a, int b) { return s[a] + o[a] < s[b] + o[b]; });", "test_policies", False),
 ]
@@ -113,7 +117,7 @@ def test_pin_catches_planted_mistake(tmp_path, source, what, old, new, pin, need
     mutated = tmp_path / "oracle_mut.cpp"
     mutated.write_text(source.replace(old, new))
     so = tmp_path / "liboracle_mut.so"
-    subprocess.check_call(["g++", "-O1", "-std=c++17", "-shared", "-fPIC", "-o", str(so), str(mutated)])
+    subprocess.check_call(["g++", "-O1", "-std=c++17", "-pthread", "-shared", "-fPIC", "-o", str(so), str(mutated)])
     root = os.path.dirname(HERE)
     r = subprocess.run([sys.executable, "-c", _CHILD, root, str(so), pin, "1" if needs_golden else "0"],
                        capture_output=True, text=True, timeout=600)

@@ -79,7 +79,7 @@ def test_example1_sorted_f_selects_type2_first(golden):
 # ----------------------------------------------------------------------------- Example 2 (symbolic)
 @pytest.mark.parametrize("n1,s1,o1,n2,s2,o2", [(10, 8, 4, 4, 20, 10), (6, 15, 5, 3, 28, 12), (5, 10, 14, 12, 4, 6)])
 def test_example2_two_saturating_batches(n1, s1, o1, n2, s2, o2):
-    """Appendix B, Example 2: n1(s1+o1) = n2(s2+o2) = M; TEL = o1 n1 + o2 n2 + (o1 n2 | o2 n1)."""
+    """the supplement to Section 3, Example 2: n1(s1+o1) = n2(s2+o2) = M; TEL = o1 n1 + o2 n2 + (o1 n2 | o2 n1)."""
     M = n1 * (s1 + o1)
     assert M == n2 * (s2 + o2)
     s = np.array([s1] * n1 + [s2] * n2, dtype=np.int32)
@@ -103,7 +103,7 @@ def test_example2_two_saturating_batches(n1, s1, o1, n2, s2, o2):
 # ----------------------------------------------------------------------------- Theorem 1 closed form
 @pytest.mark.parametrize("root4", [3, 6, 9])
 def test_theorem1_closed_form(root4, golden):
-    """Appendix A: X = M requests (sqrt(M)-1, 1) then Y = M^1.25 requests (1, 2), shortest output first."""
+    """the supplement to Section 2: X = M requests (sqrt(M)-1, 1) then Y = M^1.25 requests (1, 2), shortest output first."""
     M = root4 ** 4
     r = root4 ** 2
     X, Y = M, root4 ** 5
@@ -123,7 +123,7 @@ def test_theorem1_closed_form(root4, golden):
 
 # ----------------------------------------------------------------------------- NP-hardness family
 def test_three_partition_family(golden):
-    """Appendix A: s_i = x_i, o_i = 1, M = T + 3; optimum 3m(m+1)/2 iff a 3-partition exists."""
+    """the supplement to Section 2: s_i = x_i, o_i = 1, M = T + 3; optimum 3m(m+1)/2 iff a 3-partition exists."""
     T = 20
     x = [6, 7, 7, 6, 6, 8]                                # {6,7,7}, {6,6,8}
     s, o = np.array(x, dtype=np.int32), np.ones(6, dtype=np.int32)
@@ -254,6 +254,36 @@ def test_phase1_dp_matches_enumeration_and_lemma1():
         assert 2 * int(o[ca].sum()) > int(o[ca].max()) * len(ca)
         # the Algorithm-1 batch really is feasible when started together
         assert orc.check_schedule(s[ca], o[ca], M, np.zeros(len(ca)))["feasible"]
+
+
+def test_phase1_algorithm1_constraint_by_hand():
+    """Algorithm 1's own Phase-1 constraint, M(X, o_j) <= M for every j with all of X started
+    together, against the memory test sum(s+o) <= M of Algorithms 2-4, on an instance worked by hand.
+    A = B = (s 1, o 4), C = (s 4, o 2), M = 12.  All three started together use 3 + 3 + 6 = 12 when
+    C ends and 5 + 5 = 10 when A and B end: feasible by Algorithm 1's constraint although
+    sum(s+o) = 16 > 12.  F: {A,B,C} 10/9, {A,C} = {B,C} 6/4, {A,B} 8/4, {C} 2, {A} = {B} 4."""
+    s, o, ids = np.array([1, 1, 4]), np.array([4, 4, 2]), np.arange(3)
+    chosen, so, mem = orc.phase1_enumerate(ids, s, o, 12, orc.ENUM_ALG1)
+    assert (chosen.tolist(), so, mem) == ([0, 1, 2], 10, 16)
+    assert orc.check_schedule(s, o, 12, [0, 0, 0])["feasible"]
+    # the sum reading cannot take all three: best F among its feasible sets is 6/4, lowest indices first
+    chosen, so, mem = orc.phase1_enumerate(ids, s, o, 12, orc.ENUM_SUM)
+    assert (chosen.tolist(), so, mem) == ([0, 2], 6, 11)
+    # one token less and the round in which C ends overflows (12 > 11): Algorithm 1's constraint now
+    # refuses the triple as well, so the constraint is neither too lax nor too strict
+    assert not orc.check_schedule(s, o, 11, [0, 0, 0])["feasible"]
+    chosen, so, mem = orc.phase1_enumerate(ids, s, o, 11, orc.ENUM_ALG1)
+    assert (chosen.tolist(), so, mem) == ([0, 2], 6, 11)
+    # the later completion binds instead: A = (s 5, o 3), B = (s 6, o 3), C = (s 1, o 1), M = 17.
+    # Together: 6 + 7 + 2 = 15 when C ends, 8 + 9 = 17 when A and B end -> feasible; at M = 16 not.
+    s, o = np.array([5, 6, 1]), np.array([3, 3, 1])
+    chosen, so, _ = orc.phase1_enumerate(ids, s, o, 17, orc.ENUM_ALG1)
+    assert (chosen.tolist(), so) == ([0, 1, 2], 7)                  # F = 7/9 beats {C} = 1 and {A,C} = 4/4
+    chosen, so, _ = orc.phase1_enumerate(ids, s, o, 16, orc.ENUM_ALG1)
+    assert (chosen.tolist(), so) == ([0, 2], 4)                     # {A,C}: 6 + 2 = 8, then 8; F = 1, larger than {C}
+    # Sorted-F assembled on the first instance: the triple is one batch, sorted by o
+    order, offs = orc.sorted_f_exact(np.array([1, 1, 4]), np.array([4, 4, 2]), 12, orc.ENUM_ALG1)
+    assert order.tolist() == [2, 0, 1] and offs.tolist() == [0, 3]
 
 
 def test_sorted_f_orders_are_permutations_and_batches_sorted():
@@ -411,7 +441,7 @@ def test_workloads_are_deterministic_and_shaped():
     assert t.n == 16 and t.s.min() >= 1 and t.s.max() <= 32 and t.o.min() >= 1 and t.o.max() <= 32
 
 
-# ----------------------------------------------------------------------------- Algorithm 4 (Local Swap Search)
+# ----------------------------------------------------------------------------- Algorithm 3 (Local Swap Search)
 def test_local_swap_worked_by_hand():
     # A(1,5) B(2,5) C(5,3) D(8,1) E(9,1); sizes 6,7,8,9,10; M = 14.
     # First fit: A, B (mem 13).  out=A: C,D,E all overflow.  out=B: C fits exactly (14) and has the
@@ -500,7 +530,7 @@ def test_sorted_g_reduces_to_f_and_differs_by_hand():
     s, o = np.array([30, 1, 1], dtype=np.int32), np.array([1, 4, 4], dtype=np.int32)
     assert orc.sorted_g_prefix(s, o, 41, 0, 1)[1].tolist() == [0, 3]
     assert orc.sorted_g_prefix(s, o, 41, 1, 1)[1].tolist() == [0, 2, 3]
-    # Algorithm 4 under G: swapping in the long prompt A(30,1) for B lowers sum(o) but not sum(s+o)
+    # Algorithm 3 under G: swapping in the long prompt A(30,1) for B lowers sum(o) but not sum(s+o)
     s, o = np.array([1, 1, 3], dtype=np.int32), np.array([4, 4, 1], dtype=np.int32)      # sizes 5, 5, 4; M = 9
     assert sorted(orc.sorted_f_local_swap(s, o, 9)[0][:2].tolist()) == [0, 2]            # first fit {2,0}; nothing better
     s, o = np.array([1, 1, 4], dtype=np.int32), np.array([4, 4, 1], dtype=np.int32)      # sizes 5, 5, 5; M = 10
@@ -509,7 +539,7 @@ def test_sorted_g_reduces_to_f_and_differs_by_hand():
 
 
 # ---------------------------------------------------------------------------------------------
-# Algorithm 5 (Quantile Greedy Selection)
+# Algorithm 4 (Quantile Greedy Selection)
 # ---------------------------------------------------------------------------------------------
 def test_mix64_is_splitmix64():
     # first three outputs of splitmix64 seeded with 0 (Steele, Lea, Flood; the generator's
@@ -658,7 +688,7 @@ def test_online_with_everything_present_at_time_zero_is_the_offline_model():
             p, tot = orc.online_schedule(a, s, o, M, pol)
             rp, rtel, _ = orc.list_schedule_alg1(s, o, M, orc.policy_order(s, o, pol))
             assert (p == rp).all() and tot == rtel
-        # one planning pass over the whole backlog, never repeated: Sorted-F with Algorithm 4
+        # one planning pass over the whole backlog, never repeated: Sorted-F with Algorithm 3
         p, tot = orc.online_schedule(a, s, o, M, orc.SORTED_F, period=1 << 30, lookahead=n)
         order = orc.sorted_f_local_swap(s, o, M)[0]
         rp, rtel, _ = orc.list_schedule_alg1(s, o, M, order)
@@ -736,7 +766,7 @@ def test_sorted_f_online_worked_by_hand():
     assert p3[2] == 0 and p3[1] == 0 and p3[0] > 0
     # Example B (look-ahead 10): r0 = (0, 5, 4), r1 = (0, 6, 3), r2 = (0, 6, 2), r3 = (0, 7, 2),
     # r4 = (1, 1, 1).  First plan: batches {r2}, {r3}, {r1}, {r0} (each is alone: two never fit;
-    # Algorithm 4 walks to the shortest decode).  r2 starts in iteration 1; r3 is refused in
+    # Algorithm 3 walks to the shortest decode).  r2 starts in iteration 1; r3 is refused in
     # iterations 1 and 2 (rounds 1, 2 hold 7, 8); r4 arrives in iteration 2 and waits at the tail
     # although it would fit (8 + 2).
     a, s, o = [0, 0, 0, 0, 1], [5, 6, 6, 7, 1], [4, 3, 2, 2, 1]
@@ -759,7 +789,7 @@ def test_online_overload_ranking_of_the_three_policies():
 
 
 # ---------------------------------------------------------------------------------------------
-# Sorted-F + A_min (Section 5.5, Algorithm 6): executor under lower-bound predictions
+# Sorted-F + A_min (Section 5.5, Algorithm 5): executor under lower-bound predictions
 # ---------------------------------------------------------------------------------------------
 def test_amin_with_exact_predictions_is_algorithm_1():
     rng = np.random.default_rng(101)
