@@ -352,6 +352,22 @@ enum {
 };
 int sched_probe_peaks(double* out, int32_t n_out, int32_t repeats, void* cuda_stream);
 
+/* Which build this library is: 0, or SCHED_BUILD_CHECKED for the checked build
+ * (libkvsched_checked.so, compiled with -DKVSCHED_CHECKED), in which every index a kernel derives
+ * from data or from its own arithmetic is range-checked before use.  An index outside its array is
+ * recorded, element 0 is accessed in its place -- no access ever leaves an array, nothing traps --
+ * and the host call that next reads the device status returns SCHED_E_INTERNAL with the site
+ * number and the index in sched_last_cuda_error().  The checked build is several times slower; it
+ * is the library's own memory checker, meant to be run over small cases. */
+#define SCHED_BUILD_CHECKED 1
+int sched_build_flags(void);
+
+/* Test support for the checked build: passes `index` through the same range check against
+ * 0 .. limit-1 inside a one-thread kernel and reports as any other call would: SCHED_OK if it was in
+ * range, SCHED_E_INTERNAL (cleared afterwards) if not.  SCHED_E_UNSUPPORTED in the normal build.
+ * Nothing is accessed out of range in either case. */
+int sched_debug_check_index(int64_t index, int64_t limit);
+
 /* Test support (the paper has no counterpart): every device loop of this library whose trip count
  * depends on the data is bounded by a cap that it can never reach on valid input; a loop that does
  * reach its cap records that in a status word and returns, the kernel ends normally, and the host

@@ -12,7 +12,10 @@ import os
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libkvsched.so")
+# KVSCHED_CHECKED=1 selects the checked build of the library (every kernel index range-checked)
+CHECKED = os.environ.get("KVSCHED_CHECKED") == "1"
+LIB_PATH = os.path.join(_HERE, "libkvsched_checked.so" if CHECKED else "libkvsched.so")
+BUILD_CHECKED = 1
 
 OK, E_INVAL, E_NOT_PERMUTATION, E_CUDA, E_NOMEM, E_INTERNAL, E_UNSUPPORTED = 0, -1, -2, -3, -4, -5, -6
 CAND_ORDER, CAND_MOVE, CAND_START_TIMES, CAND_POLICY = 0, 1, 2, 3
@@ -22,7 +25,7 @@ NBHD_SWAP, NBHD_SWAP_INSERT, NBHD_SAMPLED = 0, 1, 2
 EXPORTS = [
     "sched_init", "sched_init_batch", "sched_set_stream", "sched_sync", "sched_set_prefill_weight", "sched_set_base_order",
     "sched_get_base_order", "sched_eval_batch", "sched_eval_batch_dev", "sched_sweep_dev",
-    "sched_sorted_f", "sched_sorted_f_dev", "sched_sorted_f_local_swap", "sched_sorted_f_local_swap_dev", "sched_sorted_f_dp", "sched_sorted_f_quantile", "sched_online_simulate", "sched_amin_simulate", "sched_sorted_f_amin", "sched_local_search", "sched_accept_move", "sched_last_eval_kernel_ms", "sched_argmin_static_dev", "sched_probe_peaks", "sched_debug_set_loop_cap", "sched_release_cached_memory", "sched_stats", "sched_destroy",
+    "sched_sorted_f", "sched_sorted_f_dev", "sched_sorted_f_local_swap", "sched_sorted_f_local_swap_dev", "sched_sorted_f_dp", "sched_sorted_f_quantile", "sched_online_simulate", "sched_amin_simulate", "sched_sorted_f_amin", "sched_local_search", "sched_accept_move", "sched_last_eval_kernel_ms", "sched_argmin_static_dev", "sched_probe_peaks", "sched_build_flags", "sched_debug_check_index", "sched_debug_set_loop_cap", "sched_release_cached_memory", "sched_stats", "sched_destroy",
     "sched_strerror", "sched_last_cuda_error",
 ]
 
@@ -44,8 +47,8 @@ def load():
     if _lib is not None:
         return _lib
     if not os.path.exists(LIB_PATH):
-        raise ImportError("libkvsched.so is not built: run `python -m paper_2508_06133_b200.build` "
-                          "(needs nvcc; there is no CPU fallback)")
+        raise ImportError("%s is not built: run `python -m paper_2508_06133_b200.build` "
+                          "(needs nvcc; there is no CPU fallback)" % os.path.basename(LIB_PATH))
     try:
         import torch  # noqa: F401  (loads libcudart)
     except Exception:  # pragma: no cover
@@ -79,6 +82,8 @@ def load():
     lib.sched_argmin_static_dev.argtypes = [vp, i64, i64, vp, vp]
     lib.sched_probe_peaks.argtypes = [vp, i32, i32, vp]
     lib.sched_debug_set_loop_cap.argtypes = [i32]
+    lib.sched_build_flags.argtypes = []
+    lib.sched_debug_check_index.argtypes = [i64, i64]
     lib.sched_destroy.argtypes = [vp]
     lib.sched_strerror.argtypes = [C.c_int]
     lib.sched_strerror.restype = C.c_char_p
@@ -289,6 +294,17 @@ class Scheduler:
 def release_cached_memory():
     """Return the library's cached device blocks to the driver (sched_release_cached_memory)."""
     _check(load().sched_release_cached_memory(), "sched_release_cached_memory")
+
+
+def build_flags():
+    """0, or BUILD_CHECKED when the loaded library is the checked build (sched_build_flags)."""
+    return load().sched_build_flags()
+
+
+def debug_check_index(index, limit):
+    """Checked build only: run ``index`` through the kernels' range check against 0..limit-1
+    (sched_debug_check_index); raises SchedError(E_INTERNAL) if it is out of range."""
+    _check(load().sched_debug_check_index(int(index), int(limit)), "sched_debug_check_index")
 
 
 def debug_set_loop_cap(cap):

@@ -343,7 +343,7 @@ int create_common(sched_ctx** out, int B, int n, const int32_t* s, const int32_t
             if (e1 == cudaSuccess) e1 = cudaFuncSetAttribute(k3_eval_moves<N, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn);  \
             e2 = cudaFuncSetAttribute(k3_eval_orders<N, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn); \
             if (e2 == cudaSuccess) e2 = cudaFuncSetAttribute(k3_eval_orders<N, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn); \
-            e3 = cudaFuncSetAttribute(k3_eval_policy<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn); \
+            e3 = cudaFuncSetAttribute(k3_eval_policy<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn - 2048); /* 2.2 KB of static arrays */ \
             e4 = cudaFuncSetAttribute(k3_base_run<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn)
             KV_DISPATCH_SIM(h, SETATTR);
 #undef SETATTR
@@ -367,7 +367,7 @@ int ensure_base(sched_ctx* h) {
     k3_gather_table<<<(n + 255) / 256, 256, 0, h->stream>>>(h->d_tbl_id, h->d_order, n, h->d_tbl_base);
     KV_TRY(check_launch(h));
 #define RUN(N) k3_base_run<N><<<1, 32, (size_t)h->ring_cells * sizeof(int), h->stream>>>(                  \
-        h->d_tbl_base, n, h->L, (int)h->M, h->snap_stride, h->d_snap_ring, h->d_snap_hdr,            \
+        h->d_tbl_base, n, h->L, (int)h->M, h->snap_stride, h->snap_count, h->d_snap_ring, h->d_snap_hdr, \
         h->d_base_starts, h->d_base_tel, h->d_status)
     KV_DISPATCH_SIM(h, RUN);
 #undef RUN
@@ -400,7 +400,7 @@ int order_candidates(sched_ctx* h, const MoveSource& src, i64 count) {
     KV_TRY(check_launch(h));
     k4_scan_bins<<<1, 1024, 0, h->stream>>>(bins, h->n);
     KV_TRY(check_launch(h));
-    k4_scatter_by_first_pos<<<blocks, 256, 0, h->stream>>>(first_pos, count, bins, launch_order);
+    k4_scatter_by_first_pos<<<blocks, 256, 0, h->stream>>>(first_pos, h->n, count, bins, launch_order);
     KV_TRY(check_launch(h));
     return SCHED_OK;
 }
@@ -418,7 +418,7 @@ int launch_moves(sched_ctx* h, int mode, const i64* codes, i64 first, u64 seed, 
     const size_t smem = k3_smem_bytes(h, &in_smem, &tb);
     p.n = h->n; p.L = h->L; p.M = (int)h->M; p.stride = h->snap_stride;
     p.tbl_base = h->d_tbl_base; p.table_in_smem = in_smem ? 1 : 0; p.table_bytes = tb;
-    p.snap_ring = h->d_snap_ring; p.snap_hdr = h->d_snap_hdr;
+    p.snap_ring = h->d_snap_ring; p.snap_hdr = h->d_snap_hdr; p.snap_count = h->snap_count;
     p.src.mode = mode; p.src.codes = codes; p.src.first = first; p.src.seed = seed; p.src.iteration = iteration;
     p.count = count; p.tel_out = tel_out; p.tel_by_slot = by_slot ? 1 : 0; p.starts_out = starts_out;
     p.base_order = h->d_order; p.base_starts_pos = h->d_base_starts;
@@ -455,6 +455,27 @@ i64 neighbourhood_size(int n, int nb, i64 samples) {
     return nb == SCHED_NBHD_SWAP ? nsw : nb == SCHED_NBHD_SWAP_INSERT ? nsw + (i64)n * (n - 1) : samples;
 }
 
+// Checked build only: the word in which KV_IDX records the first index that left its array.  Reads
+// it after the device is idle, clears it, and turns a recorded index into SCHED_E_INTERNAL with the
+// site and value in sched_last_cuda_error().
+int read_checked_word() {
+#ifdef KVSCHED_CHECKED
+    unsigned long long w = 0ull;
+    KV_CUDA(cudaDeviceSynchronize());
+    KV_CUDA(cudaMemcpyFromSymbol(&w, kv_checked_word, sizeof(w)));
+    if (w != 0ull) {
+        const unsigned long long zero = 0ull;
+        cudaMemcpyToSymbol(kv_checked_word, &zero, sizeof(zero));
+        long long idx = (long long)(w & 0xffffffffffull);
+        if (idx & (1ll << 39)) idx -= (1ll << 40);
+        snprintf(g_last_cuda_error, sizeof(g_last_cuda_error), "checked build: index %lld outside its array at site %d",
+                 idx, (int)(w >> 40));
+        return SCHED_E_INTERNAL;
+    }
+#endif
+    return SCHED_OK;
+}
+
 int read_status(sched_ctx* h) {
     int* hp = (int*)h->h_pinned;
     KV_CUDA(cudaMemcpyAsync(hp, h->d_status, sizeof(int), cudaMemcpyDeviceToHost, h->stream));
@@ -463,8 +484,14 @@ int read_status(sched_ctx* h) {
         cudaMemsetAsync(h->d_status, 0, sizeof(int), h->stream);
         return SCHED_E_INTERNAL;
     }
-    return SCHED_OK;
+    return read_checked_word();
 }
+
+#ifdef KVSCHED_CHECKED
+__global__ void kv_check_index_probe(long long idx, long long limit, int* sink) {
+    *sink = (int)KV_IDX(idx, limit, 9999);
+}
+#endif
 
 bool is_permutation(const int32_t* a, int n, std::vector<unsigned char>& seen) {
     seen.assign(n, 0);
@@ -537,12 +564,11 @@ int sched_eval_batch_dev(sched_handle h, int kind, int64_t count, const void* ca
     if (count >= (1ll << 31)) return SCHED_E_UNSUPPORTED;
     const int n = h->n;
     if (kind == SCHED_CAND_POLICY) {
-        const size_t smem = (size_t)(n + 1) * 16 + (size_t)n * 8 + (size_t)n * 16 + (size_t)(n + 2) * 4 +
-                            (size_t)h->ring_cells * 4;
-        if (smem > (size_t)h->smem_optin - 2048) return SCHED_E_UNSUPPORTED;
+        const size_t smem = (size_t)(n + 1) * 16 + (size_t)n * 24 + (size_t)(n + 2) * 4 + (size_t)h->ring_cells * 4;
+        if (smem > (size_t)h->smem_optin - 4096) return SCHED_E_UNSUPPORTED;
         const i64 ctas = (i64)h->B * count;
         if (ctas >= (1ll << 31)) return SCHED_E_UNSUPPORTED;
-#define RUN(N) k3_eval_policy<N><<<(unsigned)ctas, 32, smem, h->stream>>>(h->d_s, h->d_o, n, h->L, (int)h->M, \
+#define RUN(N) k3_eval_policy<N><<<(unsigned)ctas, 32, smem, h->stream>>>(h->d_s, h->d_o, n, h->L, (int)h->M, h->omax, \
                                                                   (const int*)candidates, (int)count,        \
                                                                   (i64*)tel_out, starts_out, h->d_status)
         KV_CUDA(cudaEventRecord(h->ev_k3_begin, h->stream));
@@ -1088,6 +1114,7 @@ int sched_online_simulate(int32_t B, int32_t n_max, const int32_t* n_each, const
         int status = 0;
         ON_CUDA(cudaMemcpy(&status, d_status, sizeof(int), cudaMemcpyDeviceToHost));
         if (status != 0) { rc = SCHED_E_INTERNAL; break; }
+        if ((rc = read_checked_word()) != SCHED_OK) break;
         ON_CUDA(cudaMemcpy(start_out, d_start, sizeof(int) * cells, cudaMemcpyDeviceToHost));
         ON_CUDA(cudaMemcpy(latency_out, d_lat, sizeof(i64) * (size_t)B, cudaMemcpyDeviceToHost));
         if (kernel_ms_out) ON_CUDA(cudaEventElapsedTime(kernel_ms_out, e0, e1));
@@ -1180,6 +1207,7 @@ static int amin_run(int32_t B, int32_t n_max, const int32_t* n_each, const int32
         int status = 0;
         AM_CUDA(cudaMemcpy(&status, d_status, sizeof(int), cudaMemcpyDeviceToHost));
         if (status != 0) { rc = SCHED_E_INTERNAL; break; }
+        if ((rc = read_checked_word()) != SCHED_OK) break;
         AM_CUDA(cudaMemcpy(start_out, d_start, sizeof(int) * cells, cudaMemcpyDeviceToHost));
         AM_CUDA(cudaMemcpy(tel_out, d_res, sizeof(i64) * (size_t)B, cudaMemcpyDeviceToHost));
         if (evictions_out) AM_CUDA(cudaMemcpy(evictions_out, d_res + B, sizeof(i64) * (size_t)B, cudaMemcpyDeviceToHost));
@@ -1222,6 +1250,30 @@ int sched_sorted_f_amin(int32_t n, const int32_t* s, const int32_t* lower, const
         rc = amin_run(1, n, &n, s, lower, o, M, nullptr, h->d_order, start_out, tel_out, evictions_out, peak_out, nullptr);
     sched_destroy(h);
     return rc;
+}
+
+int sched_build_flags(void) {
+#ifdef KVSCHED_CHECKED
+    return SCHED_BUILD_CHECKED;
+#else
+    return 0;
+#endif
+}
+
+int sched_debug_check_index(int64_t index, int64_t limit) {
+#ifdef KVSCHED_CHECKED
+    int* sink = nullptr;
+    KV_CUDA(cudaMalloc((void**)&sink, sizeof(int)));
+    kv_check_index_probe<<<1, 1>>>((long long)index, (long long)limit, sink);
+    cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    cudaFree(sink);
+    if (e != cudaSuccess) return kv_cuda_fail(e, "kv_check_index_probe");
+    return read_checked_word();
+#else
+    (void)index; (void)limit;
+    return SCHED_E_UNSUPPORTED;
+#endif
 }
 
 int sched_debug_set_loop_cap(int32_t cap) {

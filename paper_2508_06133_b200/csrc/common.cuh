@@ -106,6 +106,25 @@ __device__ __forceinline__ int kv_lane() { return threadIdx.x & 31; }
 __device__ __forceinline__ int kv_warp_max(int v) { return __reduce_max_sync(KV_FULL, v); }
 __device__ __forceinline__ int kv_warp_min(int v) { return __reduce_min_sync(KV_FULL, v); }
 
+// Checked build (-DKVSCHED_CHECKED, libkvsched_checked.so): every index that a kernel derives from
+// data or from its own arithmetic goes through KV_IDX(index, limit, site) before it is used.  In a
+// checked build an index outside 0 .. limit-1 is recorded (site number and value, first one wins)
+// in a device word that the host reads with the status word, and element 0 is accessed instead, so
+// nothing ever leaves its array; the host call then returns SCHED_E_INTERNAL.  In the normal build
+// KV_IDX is the index itself.  (The memory checker of the toolkit is not always available; this is
+// the library's own stand-in, run over the small parity cases.)
+#ifdef KVSCHED_CHECKED
+__device__ unsigned long long kv_checked_word = 0ull;      // 0, or (site << 40) | (index & 0xffffffffff)
+__device__ __forceinline__ long long kv_checked_index(long long idx, long long limit, int site) {
+    if (idx >= 0 && idx < limit) return idx;
+    atomicCAS(&kv_checked_word, 0ull, ((unsigned long long)site << 40) | ((unsigned long long)idx & 0xffffffffffull));
+    return 0;
+}
+#define KV_IDX(idx, limit, site) kv_checked_index((long long)(idx), (long long)(limit), (site))
+#else
+#define KV_IDX(idx, limit, site) (idx)
+#endif
+
 // Every device loop whose trip count depends on data carries a cap (its natural bound by
 // construction); a loop that reaches it records KV_DEV_LOOP_CAP in the status word and leaves, and
 // the host call returns SCHED_E_INTERNAL.  kv_test_loop_cap lowers every cap at once so that a test

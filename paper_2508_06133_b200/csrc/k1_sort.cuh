@@ -83,7 +83,7 @@ k1_radix_sort_segments(u64* __restrict__ keys_a, int* __restrict__ vals_a,
             }
             __syncthreads();
             if (valid) {
-                const int dst = lo + warp_cnt[w][d] + rank;
+                const int dst = lo + (int)KV_IDX(warp_cnt[w][d] + rank, hi - lo, 701);
                 kdst[dst] = key;
                 vdst[dst] = val;
             }

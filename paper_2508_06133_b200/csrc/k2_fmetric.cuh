@@ -104,7 +104,7 @@ __device__ int k2_select_batches(const i64* P, const i64* O, int n, i64 M, int* 
         }
         a += (int)bk;
         ++nb;
-        if (tid == 0) batch_off[nb] = a;
+        if (tid == 0) batch_off[KV_IDX(nb, n + 1, 801)] = a;
     }
     return nb;
 }

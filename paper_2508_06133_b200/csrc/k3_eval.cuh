@@ -99,7 +99,7 @@ __global__ void k3_iota(int* a, int n) {
 // ------------------------------------------------------------------------------------------------
 template <class SIM>
 __global__ void __launch_bounds__(32)
-k3_base_run(const int2* __restrict__ tbl_base, int n, int L, int M, int stride,
+k3_base_run(const int2* __restrict__ tbl_base, int n, int L, int M, int stride, int snap_count,
             int* __restrict__ snap_ring, SnapHeader* __restrict__ snap_hdr,
             int* __restrict__ base_starts_pos, i64* __restrict__ base_tel, int* status) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -114,7 +114,7 @@ k3_base_run(const int2* __restrict__ tbl_base, int n, int L, int M, int stride,
         for (int k = 0; k < cnt; ++k) {
             const int q = q0 + k;
             if (q % stride == 0) {
-                const int idx = q / stride;
+                const int idx = (int)KV_IDX(q / stride, snap_count, 401);
                 sim.store(snap_ring + (size_t)idx * L, snap_hdr + idx, lane);
             }
             const int s = __shfl_sync(KV_FULL, so.x, k), o = __shfl_sync(KV_FULL, so.y, k);
@@ -129,7 +129,7 @@ k3_base_run(const int2* __restrict__ tbl_base, int n, int L, int M, int stride,
 // Moves.  mode 0: codes[c]; mode 1: code = first + c; mode 2: sampled move m = first + c.
 // ------------------------------------------------------------------------------------------------
 struct MoveEvalParams {
-    int n, L, M, stride;
+    int n, L, M, stride, snap_count;
     const int2* tbl_base;
     int table_in_smem;
     unsigned table_bytes;              // multiple of 16
@@ -167,7 +167,7 @@ k3_eval_moves(const MoveEvalParams p) {
     const int n = p.n, L = p.L, M = p.M;
     const i64 slot = (i64)blockIdx.x * (blockDim.x >> 5) + warp;
     if (slot >= p.count) return;
-    const i64 c = p.launch_order[slot];
+    const i64 c = KV_IDX(p.launch_order[slot], p.count, 402);
     i64* tel_dst = p.tel_out + (p.tel_by_slot ? slot : c);
     SIM sim;
     sim.attach((int*)(smem_raw + ring_off) + (size_t)warp * SIM::ring_cells(L), L);
@@ -177,19 +177,19 @@ k3_eval_moves(const MoveEvalParams p) {
         return;
     }
     const int first_pos = min(mv.i, mv.j);
-    const int idx = first_pos / p.stride;
+    const int idx = (int)KV_IDX(first_pos / p.stride, p.snap_count, 403);
     const int q_start = idx * p.stride;
     // restore the base run's state in front of q_start
     sim.load(p.snap_ring + (size_t)idx * L, p.snap_hdr[idx], lane);
     int* starts = kStarts ? p.starts_out + (size_t)c * n : nullptr;
     if (kStarts)
-        for (int q = lane; q < q_start; q += 32) starts[p.base_order[q]] = p.base_starts_pos[q];
+        for (int q = lane; q < q_start; q += 32) starts[KV_IDX(p.base_order[q], n, 406)] = p.base_starts_pos[q];
     for (int q0 = q_start; q0 < n; q0 += 32) {
         const int qq = q0 + lane;
         int2 so = make_int2(1, 1);
         int id = 0;
         if (qq < n) {
-            const int bp = kv_map_pos(mv, qq);
+            const int bp = (int)KV_IDX(kv_map_pos(mv, qq), n, 404);
             so = tbl[bp];
             if (kStarts) id = p.base_order[bp];
         }
@@ -197,7 +197,7 @@ k3_eval_moves(const MoveEvalParams p) {
         for (int k = 0; k < cnt; ++k) {
             const int s = __shfl_sync(KV_FULL, so.x, k), o = __shfl_sync(KV_FULL, so.y, k);
             const int pstart = sim.admit(s, o, M, lane, p.status);
-            if (kStarts && lane == k) starts[id] = pstart;
+            if (kStarts && lane == k) starts[KV_IDX(id, n, 405)] = pstart;
         }
     }
     if (lane == 0) *tel_dst = sim.total();
@@ -263,25 +263,67 @@ k3_eval_orders(const OrderEvalParams p) {
 // ------------------------------------------------------------------------------------------------
 // Policy sweep: grid = B * P single-warp CTAs; CTA (b, k) evaluates instance b under policies[k].
 // Dynamic shared memory: the simulator's ring (SIM::ring_cells(L) ints); i64 P[n+1],
-// O[n+1]; u64 key[n]; int s[n], o[n], ord[n], tmp[n], boff[n+2].
+// O[n+1]; int s[n], o[n], three id buffers [n], batch numbers [n], boff[n+2].  Orders are built by
+// a single-warp radix sort (k3_warp_radix_sort) on the fields of the policy's key.
 // ------------------------------------------------------------------------------------------------
-__device__ __forceinline__ void k3_rank_sort(const u64* key, const int* ids_in, int* ids_out, int lo, int hi, int lane) {
-    // ids_out[lo + rank] = ids_in[e]; rank by (key, position) -- keys carry their own tie-breakers
-    for (int e = lo + lane; e < hi; e += 32) {
-        const u64 ke = key[e];
-        int rank = 0;
-        for (int f = lo; f < hi; ++f) {
-            const u64 kf = key[f];
-            rank += (kf < ke || (kf == ke && f < e)) ? 1 : 0;
+// One pass of a stable least-significant-digit radix sort run by a single warp on shared memory:
+// the m ids of `in` are written to `out` in ascending order of digit(id), an 8-bit value; ids with
+// equal digits keep their order.  `hist` is 256 ints of shared memory.  Every chunk of 32 ids is
+// ranked with a match-any vote (lanes with the same digit form a group whose lowest lane books the
+// group's bins), so no atomics are needed and the result does not depend on timing.
+template <class DIGIT>
+__device__ __forceinline__ void k3_warp_radix_pass(const int* in, int* out, int m, int* hist, int lane, DIGIT digit) {
+    for (int b = lane; b < 256; b += 32) hist[b] = 0;
+    __syncwarp();
+    const unsigned lt = (1u << lane) - 1u;
+    for (int e = lane; e < m; e += 32) atomicAdd(&hist[KV_IDX(digit(in[e]), 256, 901)], 1);   // count (order-free)
+    __syncwarp();
+    {                                                                // exclusive scan of the 256 bins, 8 per lane
+        int v[8], sum = 0;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) { v[k] = hist[8 * lane + k]; sum += v[k]; }
+        int incl = sum;
+        for (int dlt = 1; dlt < 32; dlt <<= 1) {
+            const int y = __shfl_up_sync(KV_FULL, incl, dlt);
+            if (lane >= dlt) incl += y;
         }
-        ids_out[lo + rank] = ids_in[e];
+        int run = incl - sum;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) { hist[8 * lane + k] = run; run += v[k]; }
     }
     __syncwarp();
+    for (int base = 0; base < m; base += 32) {                       // scatter
+        const int e = base + lane;
+        const int id = e < m ? in[e] : 0;
+        const int d = e < m ? digit(id) : 256 + lane;
+        const unsigned peers = __match_any_sync(KV_FULL, d);
+        int pos = 0;
+        if (e < m) pos = (int)KV_IDX(hist[KV_IDX(d, 256, 902)] + __popc(peers & lt), m, 903);
+        __syncwarp();
+        if (e < m) {
+            out[pos] = id;
+            if ((peers & lt) == 0) hist[d] += __popc(peers);
+        }
+        __syncwarp();
+    }
 }
+
+// The m ids of `a` stably re-ordered by ascending field(id) (`bytes` 8-bit digits, least significant
+// first).  a and b are two id buffers of m ints; returns the one that holds the result.
+template <class FIELD>
+__device__ __forceinline__ int* k3_warp_radix_sort(int* a, int* b, int m, int* hist, int lane, FIELD field, int bytes) {
+    for (int k = 0; k < bytes; ++k) {
+        k3_warp_radix_pass(a, b, m, hist, lane, [&](int id) { return (field(id) >> (8 * k)) & 255; });
+        int* x = a; a = b; b = x;
+    }
+    return a;
+}
+
+__host__ __device__ __forceinline__ int k3_bytes_of(unsigned v) { int b = 1; while (v >> (8 * b) && b < 4) ++b; return b; }
 
 template <class SIM>
 __global__ void __launch_bounds__(32)
-k3_eval_policy(const int* __restrict__ s_all, const int* __restrict__ o_all, int n, int L, int M,
+k3_eval_policy(const int* __restrict__ s_all, const int* __restrict__ o_all, int n, int L, int M, int omax,
                const int* __restrict__ policies, int num_policies,
                i64* __restrict__ tel_out, int* __restrict__ starts_out, int* status) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -291,54 +333,57 @@ k3_eval_policy(const int* __restrict__ s_all, const int* __restrict__ o_all, int
     int* ring = (int*)smem_raw;                       // first: 16-byte aligned for the vector loads
     i64* P = (i64*)(ring + SIM::ring_cells(L));       // a multiple of 4
     i64* O = P + (n + 1);
-    u64* key = (u64*)(O + (n + 1));
-    int* s = (int*)(key + n);
+    int* s = (int*)(O + (n + 1));
     int* o = s + n;
-    int* ord = o + n;
-    int* tmp = ord + n;
-    int* boff = tmp + n;
+    int* bufa = o + n;
+    int* bufb = bufa + n;
+    int* byo = bufb + n;                              // ids by ascending (o, id) (Sorted-F keeps them for its second sort)
+    int* bat = byo + n;                               // batch number of every request (Sorted-F)
+    int* boff = bat + n;                              // n + 2 batch offsets
     __shared__ i64 sh_warp[64];
     __shared__ i64 carry[2];
-    __shared__ u64 sh_best[66];
+    __shared__ u64 sh_best[2];                        // one warp: k2_select_batches needs no cross-warp words
+    __shared__ int hist[256];
 
     for (int i = lane; i < n; i += 32) {
         s[i] = s_all[(size_t)b * n + i];
         o[i] = o_all[(size_t)b * n + i];
-        tmp[i] = i;
+        bufa[i] = i;
     }
     __syncwarp();
-    if (policy == SCHED_POLICY_FCFS) {
-        for (int i = lane; i < n; i += 32) ord[i] = i;
+    const int o_bytes = k3_bytes_of((unsigned)omax), t_bytes = k3_bytes_of((unsigned)M);
+    auto f_o = [&](int id) { return o[id]; };
+    auto f_t = [&](int id) { return s[id] + o[id]; };
+    int* ord = bufa;                                  // FCFS: the identity order
+    // every sort is a chain of stable passes from the identity order, so ties end in ascending id
+    if (policy == SCHED_POLICY_SOF) {
+        ord = k3_warp_radix_sort(bufa, bufb, n, hist, lane, f_o, o_bytes);
+    } else if (policy == SCHED_POLICY_TOTAL_SIZE) {
+        ord = k3_warp_radix_sort(bufa, bufb, n, hist, lane, f_t, t_bytes);
+    } else if (policy == SCHED_POLICY_SORTED_F) {
+        // ascending (s+o, o, id) = the (o, id) order re-sorted stably by s+o; F-metric batch boundaries;
+        // then every batch by ascending (o, id) = the (o, id) order re-sorted stably by batch number
+        ord = k3_warp_radix_sort(bufa, bufb, n, hist, lane, f_o, o_bytes);
+        for (int i = lane; i < n; i += 32) byo[i] = ord[i];
         __syncwarp();
-    } else {
-        for (int i = lane; i < n; i += 32) {
-            const u64 T = (u64)(s[i] + o[i]), Ov = (u64)o[i];
-            key[i] = policy == SCHED_POLICY_SOF ? (Ov << 32)
-                   : policy == SCHED_POLICY_TOTAL_SIZE ? (T << 32) : ((T << 32) | Ov);
-        }
+        int* other = ord == bufa ? bufb : bufa;
+        ord = k3_warp_radix_sort(ord, other, n, hist, lane, f_t, t_bytes);
+        k2_prefix_sums(s, o, ord, n, P, O, sh_warp, carry);
         __syncwarp();
-        k3_rank_sort(key, tmp, ord, 0, n, lane);
-        if (policy == SCHED_POLICY_SORTED_F) {
-            k2_prefix_sums(s, o, ord, n, P, O, sh_warp, carry);
-            __syncwarp();
-            const int nb = k2_select_batches(P, O, n, (i64)M, boff, sh_best);
-            __syncwarp();
-            // inside every batch: ascending (o, request id)
-            for (int q = lane; q < n; q += 32) {
-                const int id = ord[q];
-                key[q] = ((u64)o[id] << 32) | (u64)(unsigned)id;
-                tmp[q] = id;
-            }
-            __syncwarp();
-            for (int bi = 0; bi < nb; ++bi) k3_rank_sort(key, tmp, ord, boff[bi], boff[bi + 1], lane);
-        }
+        const int nb = k2_select_batches(P, O, n, (i64)M, boff, sh_best);
+        __syncwarp();
+        for (int bi = 0; bi < nb; ++bi)
+            for (int q = boff[bi] + lane; q < boff[bi + 1]; q += 32) bat[KV_IDX(ord[KV_IDX(q, n, 904)], n, 905)] = bi;
+        __syncwarp();
+        auto f_b = [&](int id) { return bat[id]; };
+        ord = k3_warp_radix_sort(byo, ord == bufa ? bufb : bufa, n, hist, lane, f_b, k3_bytes_of((unsigned)nb));
     }
     SIM sim;
     sim.attach(ring, L);
     sim.reset(lane);
     int* starts = starts_out ? starts_out + ((size_t)b * num_policies + kpol) * n : nullptr;
     for (int q = 0; q < n; ++q) {
-        const int id = ord[q];
+        const int id = (int)KV_IDX(ord[q], n, 906);
         const int pstart = sim.admit(s[id], o[id], M, lane, status);
         if (starts && lane == 0) starts[id] = pstart;
     }

@@ -36,7 +36,7 @@ __global__ void k4_first_pos_histogram(MoveSource src, int n, i64 count, int* __
     int fp = min(m.i, m.j);
     if (fp < 0 || fp >= n) fp = n - 1;               // invalid code: the evaluator rejects it, any bucket will do
     first_pos[c] = fp;
-    atomicAdd(&bins[fp], 1);
+    atomicAdd(&bins[KV_IDX(fp, n, 501)], 1);
 }
 
 // exclusive scan of bins[0..n) in place (one CTA; n is at most a few hundred thousand)
@@ -65,10 +65,10 @@ __global__ void __launch_bounds__(1024) k4_scan_bins(int* __restrict__ bins, int
     }
 }
 
-__global__ void k4_scatter_by_first_pos(const int* __restrict__ first_pos, i64 count, int* __restrict__ bins,
+__global__ void k4_scatter_by_first_pos(const int* __restrict__ first_pos, int n, i64 count, int* __restrict__ bins,
                                         int* __restrict__ launch_order) {
     const i64 c = (i64)blockIdx.x * blockDim.x + threadIdx.x;
     if (c >= count) return;
-    const int slot = atomicAdd(&bins[first_pos[c]], 1);
-    launch_order[slot] = (int)c;
+    const int slot = atomicAdd(&bins[KV_IDX(first_pos[c], n, 502)], 1);
+    launch_order[KV_IDX(slot, count, 503)] = (int)c;
 }

@@ -225,7 +225,7 @@ __global__ void __launch_bounds__(K6_THREADS) k6_online(const OnlineParams P) {
             need = k6_window_need(ring, mask, t, s, o, M, sh.red);
             if (need > 0) break;
             for (int x = tid; x < o; x += K6_THREADS) ring[(t + x) & mask] += s + 1 + x;
-            if (tid == 0) P.start_out[base + r] = t - 1;
+            if (tid == 0) P.start_out[base + KV_IDX(r, n, 1001)] = t - 1;
             latency += (i64)(t - 1) + o - sa[r];
             --remaining;
             if (P.policy == SCHED_POLICY_FCFS) ++fcfs_next;

@@ -307,7 +307,7 @@ __global__ void __launch_bounds__(K7_THREADS) k7_amin(const AminParams P) {
     __syncthreads();
     u64 part = 0;
     for (int q = tid; q < n; q += K7_THREADS) {
-        P.start_out[base + pid[q]] = pp[q];
+        P.start_out[base + KV_IDX(pid[q], n, 1101)] = pp[q];
         part += (u64)((i64)pp[q] + po[q]);
     }
     if (part) atomicAdd(&acc, part);

@@ -44,11 +44,11 @@ struct SimState {
 __device__ __forceinline__ int kv_wrap(int idx, int L) {   // idx < 3L
     if (idx >= L) idx -= L;
     if (idx >= L) idx -= L;
-    return idx;
+    return (int)KV_IDX(idx, L, 301);
 }
 
 __device__ __forceinline__ int kv_wrap1(int idx, int L) {  // idx < 2L
-    return idx >= L ? idx - L : idx;
+    return (int)KV_IDX(idx >= L ? idx - L : idx, L, 302);
 }
 
 __device__ __forceinline__ void sim_reset(int* ring, int L, SimState& st, int lane) {

@@ -41,7 +41,7 @@ struct HybSim {
         fb = 0;
     }
     __device__ __forceinline__ i64 total() const { return tel; }
-    __device__ __forceinline__ int slot_of(int k) const { const int x = fb + k; return x >= FC ? x - FC : x; }
+    __device__ __forceinline__ int slot_of(int k) const { const int x = fb + k; return (int)KV_IDX(x >= FC ? x - FC : x, FC, 201); }
 
     __device__ __forceinline__ void reset(int lane) {
 #pragma unroll
@@ -51,16 +51,16 @@ struct HybSim {
     }
     __device__ __forceinline__ void load(const int* __restrict__ snap, const SnapHeader& h, int lane) {
 #pragma unroll
-        for (int c = 0; c < NREG; ++c) R[c] = snap[32 * c + lane];
-        for (int k = 0; k < FC; ++k) far[32 * k] = snap[32 * (NREG + k) + lane];
+        for (int c = 0; c < NREG; ++c) R[c] = snap[KV_IDX(32 * c + lane, span, 202)];
+        for (int k = 0; k < FC; ++k) far[32 * k] = snap[KV_IDX(32 * (NREG + k) + lane, span, 203)];
         fb = 0;
         t = h.t; tm = t & 31; rl = lane - tm;
         tel = ((i64)h.tel_hi << 32) | (i64)(unsigned)h.tel_lo;
     }
     __device__ __forceinline__ void store(int* __restrict__ snap, SnapHeader* hdr, int lane) const {
 #pragma unroll
-        for (int c = 0; c < NREG; ++c) snap[32 * c + lane] = R[c];
-        for (int k = 0; k < FC; ++k) snap[32 * (NREG + k) + lane] = far[32 * slot_of(k)];
+        for (int c = 0; c < NREG; ++c) snap[KV_IDX(32 * c + lane, span, 204)] = R[c];
+        for (int k = 0; k < FC; ++k) snap[KV_IDX(32 * (NREG + k) + lane, span, 205)] = far[32 * slot_of(k)];
         if (lane == 0) {
             SnapHeader h; h.t = t; h.hz = 0;
             h.tel_lo = (int)(tel & 0xffffffffll); h.tel_hi = (int)(tel >> 32);
@@ -74,7 +74,7 @@ struct HybSim {
         const int first = R[0];
 #pragma unroll
         for (int c = 0; c + 1 < NREG; ++c) R[c] = R[c + 1];
-        int* cell = far + 32 * fb;
+        int* cell = far + 32 * KV_IDX(fb, FC, 206);
         R[NREG - 1] = *cell;
         *cell = first;
         fb = fb + 1 == FC ? 0 : fb + 1;
@@ -82,7 +82,7 @@ struct HybSim {
 
     __device__ __forceinline__ void advance(int delta, int lane) {
         const int step = min(delta, 32 - tm);
-        if (rl >= 0 && rl < step) R[0] = t + rl + span;
+        if ((unsigned)rl < (unsigned)step) R[0] = t + rl + span;
         t += step;
         delta -= step;
         if (tm + step == 32) {
@@ -109,7 +109,7 @@ struct HybSim {
     }
     template <int KLO, int KHI>
     __device__ __forceinline__ void pass_add(int rl, int ol, int k0) {
-        if (rl >= 0 && ol > 0) R[0] = R[0] + k0;
+        if ((unsigned)rl < (unsigned)(ol + rl)) R[0] = R[0] + k0;     // 0 <= rl < o in one compare
 #pragma unroll
         for (int c = 1; c < KHI; ++c)
             if (c < KLO || 32 * c < ol) R[c] = R[c] + (k0 + 32 * c);
@@ -134,7 +134,7 @@ struct HybSim {
         int kadm = s + 1 - M - t;                      // V + kadm > 0  <=>  the cell is over budget
         for (int guard = 0;; ++guard) {
             const int ol = o - rl;
-            const int v0 = (rl >= 0 && ol > 0) ? R[0] : -1;
+            const int v0 = (unsigned)rl < (unsigned)o ? R[0] : -1;        // 0 <= rl < o: the cell is in the window
             int delta = kv_warp_max(__viaddmin_s32(v0, kadm, rl + 1));
             if (delta <= 0) {
                 const int nch = (tm + o + 31) >> 5;

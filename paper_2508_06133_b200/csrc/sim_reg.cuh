@@ -291,7 +291,7 @@ struct RegSim {
     // snapshot layout: kCells ints, R[c] of lane l at [32 c + l]
     __device__ __forceinline__ void load(const int* __restrict__ snap, const SnapHeader& h, int lane) {
 #pragma unroll
-        for (int c = 0; c < NREG; ++c) R[c] = snap[32 * c + lane];
+        for (int c = 0; c < NREG; ++c) R[c] = snap[KV_IDX(32 * c + lane, kCells, 101)];
         t = h.t;
         tm = t & 31; rl = lane - tm;
         tel = ((i64)h.tel_hi << 32) | (i64)(unsigned)h.tel_lo;
@@ -299,7 +299,7 @@ struct RegSim {
 
     __device__ __forceinline__ void store(int* __restrict__ snap, SnapHeader* hdr, int lane) const {
 #pragma unroll
-        for (int c = 0; c < NREG; ++c) snap[32 * c + lane] = R[c];
+        for (int c = 0; c < NREG; ++c) snap[KV_IDX(32 * c + lane, kCells, 102)] = R[c];
         if (lane == 0) {
             SnapHeader h; h.t = t; h.hz = 0;
             h.tel_lo = (int)(tel & 0xffffffffll); h.tel_hi = (int)(tel >> 32);
@@ -318,7 +318,7 @@ struct RegSim {
     // 32 c < ol (and rl >= 0 for c = 0), with ol = o - rl.
     template <int KLO, int KHI>
     __device__ __forceinline__ void pass_add(int rl, int ol, int k0) {
-        if (rl >= 0 && ol > 0) R[0] = R[0] + k0;
+        if ((unsigned)rl < (unsigned)(ol + rl)) R[0] = R[0] + k0;     // 0 <= rl < o in one compare
 #pragma unroll
         for (int c = 1; c < KHI; ++c)
             if (c < KLO || 32 * c < ol) R[c] = R[c] + (k0 + 32 * c);
@@ -328,7 +328,7 @@ struct RegSim {
     // (it is rare; as predicated moves it would cost NREG instructions on every call).
     __device__ __forceinline__ void advance(int delta, int lane) {
         const int step = min(delta, 32 - tm);
-        if (rl >= 0 && rl < step) R[0] = t + rl + kCells;
+        if ((unsigned)rl < (unsigned)step) R[0] = t + rl + kCells;
         t += step;
         delta -= step;
         if (tm + step == 32) {
@@ -378,7 +378,7 @@ struct RegSim {
         int kadm = s + 1 - M - t;                      // V + kadm > 0  <=>  the cell is over budget
         for (int guard = 0;; ++guard) {
             const int ol = o - rl;
-            const int v0 = (rl >= 0 && ol > 0) ? R[0] : -1;
+            const int v0 = (unsigned)rl < (unsigned)o ? R[0] : -1;        // 0 <= rl < o: the cell is in the window
             int need = __viaddmin_s32(v0, kadm, rl + 1);               // masked lanes: below zero
             int delta = kv_warp_max(need);
             if (delta <= 0) {
