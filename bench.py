@@ -314,12 +314,13 @@ def bench_policy_sweep(args, rank, world, local_rank):
     pairs = B * 4
     value = pairs * args.steps / (sum(step_ms) * 1e-3)
     cells = 4.0 * float(o.astype(np.int64).sum())                   # every pair simulates its whole list
-    # rank sorts in shared memory: n^2 key compares per sorted policy (3 of 4) and per-batch re-sort for Sorted-F (<= n^2)
-    sort_ops = 2.0 * B * 3 * n * n
+    # order construction: stable radix passes in shared memory (2 for shortest-decode-first, 2 for total-size-first,
+    # 5 for Sorted-F at these sizes), each a count and a scatter visit of n ids, ~3 integer operations per visit
+    sort_ops = 6.0 * B * 9 * n
     sm_load = clocks["sm_mhz"] or sm_max
     roofline = roofline_block(cells, kern_s, probe, probe_source, sm_load, hbm_gbs, 8.0 * B * n + 8.0 * pairs, None,
                               "k3_eval_policy", extra_ops=sort_ops)
-    roofline["extra_ops_note"] = "rank sorts: 2 integer operations per key compare, n^2 compares per sorted policy"
+    roofline["extra_ops_note"] = "order construction: 9 radix passes per instance x 2 visits x n ids x 3 integer operations"
     import oracle as orc
     got = tel.cpu().numpy().reshape(B, 4)
     cores = host_cores()

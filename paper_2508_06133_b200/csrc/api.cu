@@ -343,7 +343,8 @@ int create_common(sched_ctx** out, int B, int n, const int32_t* s, const int32_t
             if (e1 == cudaSuccess) e1 = cudaFuncSetAttribute(k3_eval_moves<N, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn);  \
             e2 = cudaFuncSetAttribute(k3_eval_orders<N, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn); \
             if (e2 == cudaSuccess) e2 = cudaFuncSetAttribute(k3_eval_orders<N, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn); \
-            e3 = cudaFuncSetAttribute(k3_eval_policy<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn - 2048); /* 2.2 KB of static arrays */ \
+            e3 = cudaFuncSetAttribute(k3_eval_policy<N, int>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn - 2048); /* 1.6 KB of static arrays */ \
+            if (e3 == cudaSuccess) e3 = cudaFuncSetAttribute(k3_eval_policy<N, i64>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn - 2048); \
             e4 = cudaFuncSetAttribute(k3_base_run<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn)
             KV_DISPATCH_SIM(h, SETATTR);
 #undef SETATTR
@@ -564,11 +565,18 @@ int sched_eval_batch_dev(sched_handle h, int kind, int64_t count, const void* ca
     if (count >= (1ll << 31)) return SCHED_E_UNSUPPORTED;
     const int n = h->n;
     if (kind == SCHED_CAND_POLICY) {
-        const size_t smem = (size_t)(n + 1) * 16 + (size_t)n * 24 + (size_t)(n + 2) * 4 + (size_t)h->ring_cells * 4;
+        if (n >= 65536) return SCHED_E_UNSUPPORTED;                    // ids are 16-bit inside the kernel
+        const bool narrow = (i64)n * h->M < (1ll << 31);               // prefix sums of s+o fit 32 bits
+        const size_t smem = (size_t)(n + 2) * 2 * (narrow ? 4 : 8) + (size_t)n * 8 + (size_t)(n + 2) * 4 + (size_t)n * 8 +
+                            (size_t)h->ring_cells * 4 + 16;
         if (smem > (size_t)h->smem_optin - 4096) return SCHED_E_UNSUPPORTED;
         const i64 ctas = (i64)h->B * count;
         if (ctas >= (1ll << 31)) return SCHED_E_UNSUPPORTED;
-#define RUN(N) k3_eval_policy<N><<<(unsigned)ctas, 32, smem, h->stream>>>(h->d_s, h->d_o, n, h->L, (int)h->M, h->omax, \
+#define RUN(N)                                                                                                       \
+        if (narrow) k3_eval_policy<N, int><<<(unsigned)ctas, 32, smem, h->stream>>>(h->d_s, h->d_o, n, h->L, (int)h->M, h->omax, \
+                                                                  (const int*)candidates, (int)count,        \
+                                                                  (i64*)tel_out, starts_out, h->d_status);   \
+        else k3_eval_policy<N, i64><<<(unsigned)ctas, 32, smem, h->stream>>>(h->d_s, h->d_o, n, h->L, (int)h->M, h->omax, \
                                                                   (const int*)candidates, (int)count,        \
                                                                   (i64*)tel_out, starts_out, h->d_status)
         KV_CUDA(cudaEventRecord(h->ev_k3_begin, h->stream));

@@ -32,8 +32,11 @@ __device__ __forceinline__ bool k2_f_better(u64 sumA, u64 kA, u64 sumB, u64 kB) 
 // P[0] = O[0] = 0, P[q+1] = P[q] + T(ids[q]).  Block-wide, chunked; `carry` is 2 shared words.
 // With a prefill weight alpha = a_num / a_den (Section 7's G-metric, alpha = 0 is F) the second sum
 // runs over a_num * s + a_den * o instead of o.
+// PT is the type the sums are stored in (int64, or int32 where the caller knows they fit); IT the
+// type of the ids.
+template <typename PT = i64, typename IT = int>
 __device__ void k2_prefix_sums(const int* __restrict__ s, const int* __restrict__ o,
-                               const int* __restrict__ ids, int n, i64* P, i64* O,
+                               const IT* __restrict__ ids, int n, PT* P, PT* O,
                                i64* sh_warp /* [2 * 32] */, i64* carry /* [2] */,
                                i64 a_num = 0, i64 a_den = 1) {
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5, nw = blockDim.x >> 5;
@@ -52,7 +55,7 @@ __device__ void k2_prefix_sums(const int* __restrict__ s, const int* __restrict_
         __syncthreads();
         i64 bt = carry[0], bo = carry[1];
         for (int k = 0; k < w; ++k) { bt += sh_warp[k]; bo += sh_warp[32 + k]; }
-        if (q < n) { P[q + 1] = bt + it; O[q + 1] = bo + io; }
+        if (q < n) { P[q + 1] = (PT)(bt + it); O[q + 1] = (PT)(bo + io); }
         __syncthreads();
         if (tid == blockDim.x - 1) {
             i64 tt = 0, to = 0;
@@ -65,22 +68,23 @@ __device__ void k2_prefix_sums(const int* __restrict__ s, const int* __restrict_
 
 // Batch boundaries by the rule above.  Writes batch_off[0..nb] and returns nb (same in all
 // threads).  sh_best: 2 * 32 + 2 shared 64-bit words.
-__device__ int k2_select_batches(const i64* P, const i64* O, int n, i64 M, int* batch_off, u64* sh_best) {
+template <typename PT = i64>
+__device__ int k2_select_batches(const PT* P, const PT* O, int n, i64 M, int* batch_off, u64* sh_best) {
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5, nw = blockDim.x >> 5;
     int a = 0, nb = 0;
     if (tid == 0) batch_off[0] = 0;
     while (a < n) {
         // k_max by binary search on P (every thread does the same search)
         int lo_k = 1, hi_k = n - a;
-        const i64 Pa = P[a], Oa = O[a];
+        const i64 Pa = (i64)P[a], Oa = (i64)O[a];
         while (lo_k < hi_k) {
             int mid = (lo_k + hi_k + 1) >> 1;
-            if (P[a + mid] - Pa <= M) lo_k = mid; else hi_k = mid - 1;
+            if ((i64)P[a + mid] - Pa <= M) lo_k = mid; else hi_k = mid - 1;
         }
         const int kmax = lo_k;                      // >= 1 because every request fits on its own
         u64 bs = 0, bk = 0;
         for (int k = 1 + tid; k <= kmax; k += blockDim.x) {
-            u64 sum = (u64)(O[a + k] - Oa);
+            u64 sum = (u64)((i64)O[a + k] - Oa);
             if (k2_f_better(sum, (u64)k, bs, bk)) { bs = sum; bk = (u64)k; }
         }
         for (int d = 16; d >= 1; d >>= 1) {

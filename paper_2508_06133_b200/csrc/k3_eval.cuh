@@ -262,8 +262,9 @@ k3_eval_orders(const OrderEvalParams p) {
 
 // ------------------------------------------------------------------------------------------------
 // Policy sweep: grid = B * P single-warp CTAs; CTA (b, k) evaluates instance b under policies[k].
-// Dynamic shared memory: the simulator's ring (SIM::ring_cells(L) ints); i64 P[n+1],
-// O[n+1]; int s[n], o[n], three id buffers [n], batch numbers [n], boff[n+2].  Orders are built by
+// Dynamic shared memory: the simulator's ring (SIM::ring_cells(L) ints); PT P[n+2], O[n+2] (PT =
+// int32 when n * M < 2^31, else int64); int s[n], o[n], boff[n+2]; 16-bit: three id buffers [n] and
+// batch numbers [n].  Orders are built by
 // a single-warp radix sort (k3_warp_radix_sort) on the fields of the policy's key.
 // ------------------------------------------------------------------------------------------------
 // One pass of a stable least-significant-digit radix sort run by a single warp on shared memory:
@@ -271,8 +272,8 @@ k3_eval_orders(const OrderEvalParams p) {
 // equal digits keep their order.  `hist` is 256 ints of shared memory.  Every chunk of 32 ids is
 // ranked with a match-any vote (lanes with the same digit form a group whose lowest lane books the
 // group's bins), so no atomics are needed and the result does not depend on timing.
-template <class DIGIT>
-__device__ __forceinline__ void k3_warp_radix_pass(const int* in, int* out, int m, int* hist, int lane, DIGIT digit) {
+template <class IT, class DIGIT>
+__device__ __forceinline__ void k3_warp_radix_pass(const IT* in, IT* out, int m, int* hist, int lane, DIGIT digit) {
     for (int b = lane; b < 256; b += 32) hist[b] = 0;
     __syncwarp();
     const unsigned lt = (1u << lane) - 1u;
@@ -301,7 +302,7 @@ __device__ __forceinline__ void k3_warp_radix_pass(const int* in, int* out, int 
         if (e < m) pos = (int)KV_IDX(hist[KV_IDX(d, 256, 902)] + __popc(peers & lt), m, 903);
         __syncwarp();
         if (e < m) {
-            out[pos] = id;
+            out[pos] = (IT)id;
             if ((peers & lt) == 0) hist[d] += __popc(peers);
         }
         __syncwarp();
@@ -310,18 +311,20 @@ __device__ __forceinline__ void k3_warp_radix_pass(const int* in, int* out, int 
 
 // The m ids of `a` stably re-ordered by ascending field(id) (`bytes` 8-bit digits, least significant
 // first).  a and b are two id buffers of m ints; returns the one that holds the result.
-template <class FIELD>
-__device__ __forceinline__ int* k3_warp_radix_sort(int* a, int* b, int m, int* hist, int lane, FIELD field, int bytes) {
+template <class IT, class FIELD>
+__device__ __forceinline__ IT* k3_warp_radix_sort(IT* a, IT* b, int m, int* hist, int lane, FIELD field, int bytes) {
     for (int k = 0; k < bytes; ++k) {
         k3_warp_radix_pass(a, b, m, hist, lane, [&](int id) { return (field(id) >> (8 * k)) & 255; });
-        int* x = a; a = b; b = x;
+        IT* x = a; a = b; b = x;
     }
     return a;
 }
 
 __host__ __device__ __forceinline__ int k3_bytes_of(unsigned v) { int b = 1; while (v >> (8 * b) && b < 4) ++b; return b; }
 
-template <class SIM>
+typedef unsigned short k3_id_t;                     // request ids and list positions of the policy kernel (n < 65,536)
+
+template <class SIM, typename PT>
 __global__ void __launch_bounds__(32)
 k3_eval_policy(const int* __restrict__ s_all, const int* __restrict__ o_all, int n, int L, int M, int omax,
                const int* __restrict__ policies, int num_policies,
@@ -331,16 +334,16 @@ k3_eval_policy(const int* __restrict__ s_all, const int* __restrict__ o_all, int
     const int b = blockIdx.x / num_policies, kpol = blockIdx.x % num_policies;
     const int policy = policies[kpol];
     int* ring = (int*)smem_raw;                       // first: 16-byte aligned for the vector loads
-    i64* P = (i64*)(ring + SIM::ring_cells(L));       // a multiple of 4
-    i64* O = P + (n + 1);
-    int* s = (int*)(O + (n + 1));
+    PT* P = (PT*)(ring + SIM::ring_cells(L));         // a multiple of 4 ints: 8-byte aligned
+    PT* O = P + (n + 2);
+    int* s = (int*)(O + (n + 2));
     int* o = s + n;
-    int* bufa = o + n;
-    int* bufb = bufa + n;
-    int* byo = bufb + n;                              // ids by ascending (o, id) (Sorted-F keeps them for its second sort)
-    int* bat = byo + n;                               // batch number of every request (Sorted-F)
-    int* boff = bat + n;                              // n + 2 batch offsets
-    __shared__ i64 sh_warp[64];
+    int* boff = o + n;                                // n + 2 batch offsets
+    k3_id_t* bufa = (k3_id_t*)(boff + n + 2);
+    k3_id_t* bufb = bufa + n;
+    k3_id_t* byo = bufb + n;                          // ids by ascending (o, id) (Sorted-F keeps them for its second sort)
+    k3_id_t* bat = byo + n;                           // batch number of every request (Sorted-F)
+    __shared__ i64 sh_warp[33];                       // one warp: k2_prefix_sums uses words 0 and 32
     __shared__ i64 carry[2];
     __shared__ u64 sh_best[2];                        // one warp: k2_select_batches needs no cross-warp words
     __shared__ int hist[256];
@@ -348,13 +351,13 @@ k3_eval_policy(const int* __restrict__ s_all, const int* __restrict__ o_all, int
     for (int i = lane; i < n; i += 32) {
         s[i] = s_all[(size_t)b * n + i];
         o[i] = o_all[(size_t)b * n + i];
-        bufa[i] = i;
+        bufa[i] = (k3_id_t)i;
     }
     __syncwarp();
     const int o_bytes = k3_bytes_of((unsigned)omax), t_bytes = k3_bytes_of((unsigned)M);
     auto f_o = [&](int id) { return o[id]; };
     auto f_t = [&](int id) { return s[id] + o[id]; };
-    int* ord = bufa;                                  // FCFS: the identity order
+    k3_id_t* ord = bufa;                              // FCFS: the identity order
     // every sort is a chain of stable passes from the identity order, so ties end in ascending id
     if (policy == SCHED_POLICY_SOF) {
         ord = k3_warp_radix_sort(bufa, bufb, n, hist, lane, f_o, o_bytes);
@@ -366,7 +369,7 @@ k3_eval_policy(const int* __restrict__ s_all, const int* __restrict__ o_all, int
         ord = k3_warp_radix_sort(bufa, bufb, n, hist, lane, f_o, o_bytes);
         for (int i = lane; i < n; i += 32) byo[i] = ord[i];
         __syncwarp();
-        int* other = ord == bufa ? bufb : bufa;
+        k3_id_t* other = ord == bufa ? bufb : bufa;
         ord = k3_warp_radix_sort(ord, other, n, hist, lane, f_t, t_bytes);
         k2_prefix_sums(s, o, ord, n, P, O, sh_warp, carry);
         __syncwarp();

@@ -104,7 +104,7 @@ struct HybSim {
         for (int c = 1; c + 1 < KI; c += 2) v = __vimax3_s32(v, R[c], R[c + 1]);
         if constexpr (KI >= 2 && ((KI - 1) & 1)) v = max(v, R[KI - 1]);
 #pragma unroll
-        for (int c = (KI > 1 ? KI : 1); c < KHI; ++c) v = max(v, (32 * c < ol) ? R[c] : -1);
+        for (int c = (KI > 1 ? KI : 1); c < KHI; ++c) if (32 * c < ol) v = max(v, R[c]);
         return v;
     }
     template <int KLO, int KHI>
