@@ -118,7 +118,10 @@ int sched_get_base_order(sched_handle h, int32_t* order_out);
  *   starts_out   : nullable; int32[count][n] start time p_i of every request i, indexed by request
  *                  id (ORDER, MOVE, and POLICY with layout [B][count][n_each]).
  * Host-pointer form: validates ORDER candidates (SCHED_E_NOT_PERMUTATION), MOVE codes and policy
- * ids (SCHED_E_INVAL) and negative start times (SCHED_E_INVAL) before any launch. */
+ * ids (SCHED_E_INVAL) and negative start times (SCHED_E_INVAL) before any launch.
+ * POLICY builds every order inside the kernel (one warp per instance-policy pair, all of an
+ * instance's arrays in shared memory): SCHED_E_UNSUPPORTED when the instance does not fit there
+ * (about n > 8,000 requests on a single-instance handle; batch handles are limited to 1,024). */
 int sched_eval_batch(sched_handle h, int kind, int64_t count, const void* candidates,
                      int64_t* tel_out, uint8_t* feasible_out, int32_t* starts_out);
 

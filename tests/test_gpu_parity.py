@@ -893,6 +893,27 @@ def test_a_loop_cap_that_runs_out_is_reported_and_leaves_the_handle_usable():
         assert (h.eval_batch(kv.CAND_POLICY, pols)[0] == good).all()
 
 
+def test_probe_peaks_are_plausible():
+    """The roofline denominators come from the library's own probe kernels: every rate must be positive
+    and finite, no pipe can beat the issue limit of 128 lanes per clock and SM at the top clock, the
+    integer ALU pipe alone must not beat compiler-scheduled adds, and repeated calls agree."""
+    import torch
+    prop = torch.cuda.get_device_properties(torch.cuda.current_device())
+    a = kv.probe_peaks(repeats=3)
+    b = kv.probe_peaks(repeats=3)
+    assert set(a) == set(kv.PROBE_NAMES)
+    limit = prop.multi_processor_count * 128 * 2.2e9                 # lanes x a clock no B200 reaches
+    for name in ("int_add", "int_add_max", "int_mad", "sim_mix", "int_alu"):
+        assert 0 < a[name] < limit and abs(a[name] - b[name]) < 0.1 * a[name], (name, a[name], b[name])
+    assert a["int_alu"] <= 1.05 * a["int_add"] and a["int_mad"] <= 1.05 * a["int_add"]
+    for name in ("smem_load", "smem_store"):
+        assert 0 < a[name] < prop.multi_processor_count * 256 * 2.2e9
+    lib = kv.load()
+    assert lib.sched_probe_peaks(None, 7, 3, None) == kv.E_INVAL
+    out = np.zeros(3)
+    assert lib.sched_probe_peaks(out.ctypes.data, 3, 3, None) == kv.E_INVAL
+
+
 # ------------------------------------------------------------------------------------ full-size configurations
 def test_policy_sweep_full_size_sampled_instances():
     """4,096 instances x 4 policies in one launch; a sample of instances is re-evaluated by the oracle."""

@@ -190,6 +190,28 @@ def test_alg1_equals_round_form_and_invariants():
         assert (np.diff(p1[order]) >= 0).all()
 
 
+def test_alg1_equals_round_form_on_mixed_backlogs():
+    """The same equivalence at the sizes and shapes the bulk GPU parity relies on: mixed chat/document
+    backlogs of a few hundred to 1,500 requests (saturated memory, long waits, hundreds of requests
+    running at once), under Sorted-F, the three baseline policies, random orders and moved orders --
+    every start time, not only the TEL."""
+    rng = np.random.default_rng(2024)
+    for n, M, seed in ((300, 20000, 11), (400, 24000, 12), (700, 40000, 13), (1500, 65536, 14)):
+        inst = W.mixed_backlog(n, seed, M, name="o2")
+        base, _ = orc.sorted_f_prefix(inst.s, inst.o, inst.M)
+        orders = [base, orc.policy_order(inst.s, inst.o, orc.FCFS), orc.policy_order(inst.s, inst.o, orc.SHORTEST_OUTPUT_FIRST),
+                  orc.policy_order(inst.s, inst.o, orc.TOTAL_SIZE_FIRST), rng.permutation(n).astype(np.int32)]
+        total = n * (n - 1) // 2 + n * (n - 1)
+        for code in rng.integers(0, total, 4 if n > 1000 else 8):
+            orders.append(orc.apply_move(base, *orc.decode_move(n, int(code))))
+        for order in orders:
+            p1, tel1, mk1 = orc.list_schedule_alg1(inst.s, inst.o, inst.M, order)
+            p2, tel2, mk2 = orc.list_schedule_rounds(inst.s, inst.o, inst.M, order)
+            assert (p1 == p2).all() and tel1 == tel2 and mk1 == mk2
+        chk = orc.check_schedule(inst.s, inst.o, inst.M, p1)
+        assert chk["feasible"] and chk["tel"] == tel1
+
+
 def test_each_start_is_the_earliest_feasible():
     """Break rule + maximal admission: request q starts at the first round >= its predecessor's
     start at which the occupancy definition admits it, given the earlier requests."""
