@@ -20,7 +20,7 @@ The roofline denominators are measured inside this run by the library's probe ke
 (`sched_probe_peaks`): `roofline.frac` is read against the measured rate of the integer ALU pipe (the
 pipe every maximum, compare and select of the simulator has to go through); `roofline.frac_vs` gives
 the same achieved figure against the other measured rates -- plain adds, which the compiler spreads
-over two pipes, multiply-adds, the simulator's own opcode mix -- and the instruction-issue limit.
+over two pipes, multiply-adds, a two-pipe mix -- and the instruction-issue limit.
 """
 from __future__ import annotations
 

@@ -334,7 +334,7 @@ int sched_sorted_f_amin(int32_t n, const int32_t* s, const int32_t* lower, const
  *   out[SCHED_PROBE_INT_ADD]      32-bit integer adds
  *   out[SCHED_PROBE_INT_ADD_MAX]  adds and maxima alternating
  *   out[SCHED_PROBE_INT_MAD]      32-bit integer multiply-adds
- *   out[SCHED_PROBE_SIM_MIX]      the simulator's window-pass mix: multiply-add, 3-input max, add
+ *   out[SCHED_PROBE_SIM_MIX]      a two-pipe mix: multiply-add, 3-input max, add in turn
  *   out[SCHED_PROBE_SMEM_LOAD]    shared-memory loads, 16 bytes per thread and access
  *   out[SCHED_PROBE_SMEM_STORE]   shared-memory stores, 16 bytes per thread and access
  *   out[SCHED_PROBE_INT_ALU]      maxima and exclusive-ors alternating: work that only the integer

@@ -6,8 +6,8 @@
 //   0  int32 add            a += b; b += a                       (integer ALU pipe)
 //   1  int32 add + max      a += b; b = max(b, a)                (integer ALU pipe, two opcodes)
 //   2  int32 multiply-add   a = a * k + b; b = b * k + a         (FMA pipe)
-//   3  simulator mix        one multiply-add, one 3-input max, one add per step: the opcode mix
-//                           of the register-resident simulator's window passes
+//   3  two-pipe mix         one multiply-add, one 3-input max, one add per step: one operation on
+//                           the FMA pipe for two on the integer ALU pipe
 //   4  shared-memory loads  16 bytes per thread and access, conflict-free
 //   5  shared-memory stores 16 bytes per thread and access, conflict-free
 //   6  int32 max + xor      a = max(a, b); b ^= a                (integer ALU pipe only: the compiler may
@@ -44,9 +44,9 @@ __global__ void __launch_bounds__(kThreads) probe_alu(int iters, int seed, int m
                 if (KIND == 2) { a[c] = a[c] * mul + b[c]; b[c] = b[c] * mul + a[c]; }
                 if (KIND == 6) { a[c] = max(a[c], b[c]); b[c] ^= a[c]; }
                 if (KIND == 3) {
-                    a[c] = a[c] * mul + b[c];                                   // ramp add, issued as a multiply-add
-                    b[c] = __vimax3_s32(b[c], a[c], a[(c + 1) % kChains]);      // window maximum, two cells per instruction
-                    a[c] += b[c];                                               // per-chunk constant
+                    a[c] = a[c] * mul + b[c];                                   // FMA pipe
+                    b[c] = __vimax3_s32(b[c], a[c], a[(c + 1) % kChains]);      // integer ALU pipe
+                    a[c] += b[c];                                               // either pipe
                 }
             }
         }
