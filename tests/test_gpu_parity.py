@@ -78,6 +78,37 @@ def test_orders_long_waits_and_ring_wrap():
             assert tel[c] == t and (starts[c] == p).all()
 
 
+@pytest.mark.parametrize("sim", ["", "smem", "hybrid"])
+def test_orders_wait_decided_behind_the_first_chunk(sim, monkeypatch):
+    """The simulators look at the first 32 rounds of a window before anything else.  Here the only
+    rounds over budget lie behind them: with M = 195, A = (s 100, o 40) runs from round 0 and peaks at
+    140 tokens in round 39; B = (s 20, o 60) fits beside it in rounds 0..31 (at most 132 + 52 = 184)
+    and first overflows in round 37 (138 + 58 = 196), so its wait comes from the second chunk alone.
+    Also with the pair shifted to every kind of start offset inside a chunk, with longer tails, and
+    in other orders; on the default simulator and on the two with shared-memory timelines."""
+    if sim:
+        monkeypatch.setenv("KVSCHED_SIM", sim)
+    M = 195
+    for lead in (0, 1, 5, 17, 31, 32, 33, 63):                     # a request of `lead` rounds in front moves t
+        for tail in (60, 90, 150):
+            s = np.array([50, 100, 20, 3, 7], dtype=np.int32)
+            o = np.array([max(lead, 1), 40, tail, 64, 33], dtype=np.int32)
+            n = len(s)
+            orders = np.stack([np.arange(n), np.arange(n)[::-1], np.roll(np.arange(n), 1)]).astype(np.int32)
+            with kv.Scheduler(s, o, M) as h:
+                tel, _, starts = h.eval_batch(kv.CAND_ORDER, orders, want_starts=True)
+            for c in range(len(orders)):
+                p, t, _ = orc.list_schedule_alg1(s, o, M, orders[c])
+                assert tel[c] == t and (starts[c] == p).all(), (o.tolist(), orders[c].tolist())
+    # the stated pair on its own, checked by hand: round 37 is the first over budget, and B's ramp
+    # has to drop by 196 - 195 = 1 there while A's peak (round 39: 140 + 60 = 200) asks for 5
+    s, o = np.array([100, 20], dtype=np.int32), np.array([40, 60], dtype=np.int32)
+    with kv.Scheduler(s, o, M) as h:
+        tel, _, starts = h.eval_batch(kv.CAND_ORDER, np.array([[0, 1]], dtype=np.int32), want_starts=True)
+    assert starts[0].tolist() == [0, 5] and tel[0] == 40 + 65
+    assert orc.list_schedule_alg1(s, o, M, [0, 1])[0].tolist() == [0, 5]
+
+
 @pytest.mark.parametrize("omax", [100, 127, 128, 129, 255, 256, 257, 511, 512, 513, 1023, 1024, 1025, 1500, 3000])
 def test_orders_every_simulator_shape(omax):
     """Window lengths around each register count's limit, and the hybrid simulator beyond 1025."""
