@@ -46,7 +46,8 @@ enum {
     SCHED_E_NOT_PERMUTATION = -2,  /* an ORDER candidate (or order_inout) is not a permutation of 0..n-1 */
     SCHED_E_CUDA = -3,             /* a CUDA runtime call failed (sched_last_cuda_error() has the text) */
     SCHED_E_NOMEM = -4,            /* host or device allocation failed */
-    SCHED_E_INTERNAL = -5,         /* a bounded device loop hit its cap; results are not valid */
+    SCHED_E_INTERNAL = -5,         /* a bounded device loop hit its cap (or, in the checked build, an index
+                                      left its array); results are not valid */
     SCHED_E_UNSUPPORTED = -6       /* sizes beyond what this build handles (see each call) */
 };
 

@@ -1320,7 +1320,7 @@ const char* sched_strerror(int code) {
         case SCHED_E_NOT_PERMUTATION: return "candidate is not a permutation of 0..n-1";
         case SCHED_E_CUDA: return "CUDA runtime error";
         case SCHED_E_NOMEM: return "out of memory";
-        case SCHED_E_INTERNAL: return "a bounded device loop hit its cap";
+        case SCHED_E_INTERNAL: return "a bounded device loop hit its cap, or the checked build caught an index outside its array";
         case SCHED_E_UNSUPPORTED: return "size not supported by this build";
         default: return "unknown error code";
     }
