@@ -1,4 +1,4 @@
-"""GPU parity at the stated sizes of the two large configurations.
+"""GPU parity at the stated sizes of the two large configurations, and whole sampled neighbourhoods.
 
 * n = 10,000 (the headline backlog): ONE complete swap + insert sweep of the Sorted-F order, all
   149,985,000 neighbours, through ``sched_sweep_dev`` with every TEL dumped.  The arg-min is
@@ -10,8 +10,12 @@
   2^20 sampled moves each.  Every iteration's reported (sample index, TEL) is replayed through the
   oracle's executor, and the final order must be the replay's.  Three iterations by default; the
   configuration's 50 with ``KVSCHED_FULL_CONFIGS=1`` (about a quarter of an hour of GPU time).
+* every sweep workload of the benchmark: one sampled neighbourhood with every TEL dumped and ALL of
+  them re-evaluated by the oracle (candidates split over the host's cores), plus the reduced
+  (TEL, index) pair: 16,384 / 512 / 65,536 / 65,536 moves at n = 10,000 / 100,000 / 2,000 / 1,000 by
+  default, eight times as many with ``KVSCHED_FULL_CONFIGS=1``.
 
-Both tests print one line with the wall time and the TELs (``pytest -s`` shows it).
+The tests print one line each with the wall time and the TELs (``pytest -s`` shows it).
 """
 import os
 import time
@@ -103,3 +107,34 @@ def test_heavy_100k_sampled_local_search():
     assert (final == cur).all() and ftel == cur_tel and ftel <= tel0
     print("\nheavy_100k: %d iterations x %d sampled moves in %.1f s (%.3e evals/s), %d accepted, TEL %d -> %d"
           % (iters, samples, wall, iters * samples / wall, accepted, tel0, ftel))
+
+
+@pytest.mark.parametrize("workload,moves", [("mixed_10k", 16384), ("heavy_100k", 512), ("paper_scale", 65536), ("mixed_1k", 65536)])
+def test_every_tel_of_a_sampled_neighbourhood(workload, moves):
+    import torch
+    import bench
+    if os.environ.get("KVSCHED_FULL_CONFIGS") == "1":
+        moves *= 8
+    inst = getattr(W, workload)()
+    n, seed, it = inst.n, 4242, 7
+    dev = torch.device("cuda", torch.cuda.current_device())
+    tel = torch.empty(moves, dtype=torch.int64, device=dev)
+    best = torch.zeros(2, dtype=torch.int64, device=dev)
+    base, _ = orc.sorted_f_prefix(inst.s, inst.o, inst.M)
+    with kv.Scheduler(inst.s, inst.o, inst.M) as h:
+        order, _, _ = h.sorted_f()
+        assert (order == base).all()
+        h.sweep_dev(moves, best, sampled=True, seed=seed, iteration=it, first_code=0, tel_out=tel)
+        h.sync()
+    ty, mi, mj = bench.sampled_move_positions(n, seed, it, 0, moves)      # pinned to the oracle's generator on the CPU
+    swap = (ty == 0) & (mi > mj)
+    mi, mj = np.where(swap, mj, mi), np.where(swap, mi, mj)
+    t0 = time.perf_counter()
+    ref = orc.eval_moves_threads(inst.s, inst.o, inst.M, base, ty, mi, mj, threads=bench.host_cores())
+    dt = time.perf_counter() - t0
+    got = tel.cpu().numpy()
+    assert (got == ref).all(), "%d of %d TELs differ" % (int((got != ref).sum()), moves)
+    k = int(np.argmin(ref))
+    assert best.cpu().tolist() == [int(ref[k]), k]
+    print("\n%s: %d sampled moves, every TEL equal to the oracle's (%.1f s of oracle time on %d cores)"
+          % (workload, moves, dt, bench.host_cores()))
