@@ -48,7 +48,7 @@ OPS_PER_CELL, BYTES_PER_CELL = 4.0, 8.0  # algorithmic cost of one timeline cell
 # dram__bytes_read.sum + dram__bytes_write.sum of one simulator launch, from a one-pass ncu capture of
 # this very launch (summary under profiles/); keyed by (workload, moves per launch) with a digest of
 # the simulator's source files, so that it turns into null when the kernel changes
-K3_TRAFFIC = {("mixed_n10000", 1 << 22): (60.89e6 + 9.96e6, "0b4e72470c29ccfc")}
+K3_TRAFFIC = {("mixed_n10000", 1 << 22): (61.21e6 + 10.59e6, "1e184f7ce88dd053")}
 DEFAULT_MOVES = {"mixed_10k": 1 << 22, "mixed_1k": 499500, "paper_scale": 1 << 21, "heavy_100k": 1 << 18}
 
 

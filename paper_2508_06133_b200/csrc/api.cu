@@ -17,6 +17,7 @@
 #include "k2_dp.cuh"
 #include "k2_quantile.cuh"
 #include "k3_eval.cuh"
+#include "k3_policy.cuh"
 #include "k5_argmin.cuh"
 #include "k6_online.cuh"
 #include "k7_amin.cuh"
@@ -343,7 +344,7 @@ int create_common(sched_ctx** out, int B, int n, const int32_t* s, const int32_t
             if (e1 == cudaSuccess) e1 = cudaFuncSetAttribute(k3_eval_moves<N, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn);  \
             e2 = cudaFuncSetAttribute(k3_eval_orders<N, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn); \
             if (e2 == cudaSuccess) e2 = cudaFuncSetAttribute(k3_eval_orders<N, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn); \
-            e3 = cudaFuncSetAttribute(k3_eval_policy<N, int>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn - 2048); /* 1.6 KB of static arrays */ \
+            e3 = cudaFuncSetAttribute(k3_eval_policy<N, int>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn - 2048); \
             if (e3 == cudaSuccess) e3 = cudaFuncSetAttribute(k3_eval_policy<N, i64>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn - 2048); \
             e4 = cudaFuncSetAttribute(k3_base_run<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn)
             KV_DISPATCH_SIM(h, SETATTR);
@@ -567,17 +568,23 @@ int sched_eval_batch_dev(sched_handle h, int kind, int64_t count, const void* ca
     if (kind == SCHED_CAND_POLICY) {
         if (n >= 65536) return SCHED_E_UNSUPPORTED;                    // ids are 16-bit inside the kernel
         const bool narrow = (i64)n * h->M < (1ll << 31);               // prefix sums of s+o fit 32 bits
-        const size_t smem = (size_t)(n + 2) * 2 * (narrow ? 4 : 8) + (size_t)n * 8 + (size_t)(n + 2) * 4 + (size_t)n * 8 +
-                            (size_t)h->ring_cells * 4 + 16;
-        if (smem > (size_t)h->smem_optin - 4096) return SCHED_E_UNSUPPORTED;
-        const i64 ctas = (i64)h->B * count;
+        const size_t shared_so = ((size_t)n * 8 + 15) & ~(size_t)15;
+        const size_t per_warp = k3_policy_warp_bytes(n, h->ring_cells, narrow ? 4 : 8);
+        const size_t room = (size_t)h->smem_optin - 4096;
+        if (shared_so + per_warp > room) return SCHED_E_UNSUPPORTED;
+        int W = (int)((room - shared_so) / per_warp);                  // pairs of one instance per CTA
+        if (W > K3P_MAX_WARPS) W = K3P_MAX_WARPS;
+        if ((i64)W > count) W = (int)count;
+        const int groups = (int)((count + W - 1) / W);
+        const size_t smem = shared_so + (size_t)W * per_warp;
+        const i64 ctas = (i64)h->B * groups;
         if (ctas >= (1ll << 31)) return SCHED_E_UNSUPPORTED;
 #define RUN(N)                                                                                                       \
-        if (narrow) k3_eval_policy<N, int><<<(unsigned)ctas, 32, smem, h->stream>>>(h->d_s, h->d_o, n, h->L, (int)h->M, h->omax, \
-                                                                  (const int*)candidates, (int)count,        \
+        if (narrow) k3_eval_policy<N, int><<<(unsigned)ctas, 32 * W, smem, h->stream>>>(h->d_s, h->d_o, n, h->L, (int)h->M, h->omax, \
+                                                                  (const int*)candidates, (int)count, groups, \
                                                                   (i64*)tel_out, starts_out, h->d_status);   \
-        else k3_eval_policy<N, i64><<<(unsigned)ctas, 32, smem, h->stream>>>(h->d_s, h->d_o, n, h->L, (int)h->M, h->omax, \
-                                                                  (const int*)candidates, (int)count,        \
+        else k3_eval_policy<N, i64><<<(unsigned)ctas, 32 * W, smem, h->stream>>>(h->d_s, h->d_o, n, h->L, (int)h->M, h->omax, \
+                                                                  (const int*)candidates, (int)count, groups, \
                                                                   (i64*)tel_out, starts_out, h->d_status)
         KV_CUDA(cudaEventRecord(h->ev_k3_begin, h->stream));
         KV_DISPATCH_SIM(h, RUN);
@@ -585,8 +592,8 @@ int sched_eval_batch_dev(sched_handle h, int kind, int64_t count, const void* ca
         KV_TRY(check_launch(h));
         KV_CUDA(cudaEventRecord(h->ev_k3_end, h->stream));
         h->ev_valid = true;
-        h->evaluations += ctas;
-        if (feasible_out) KV_CUDA(cudaMemsetAsync(feasible_out, 1, (size_t)ctas, h->stream));
+        h->evaluations += (i64)h->B * count;
+        if (feasible_out) KV_CUDA(cudaMemsetAsync(feasible_out, 1, (size_t)((i64)h->B * count), h->stream));
         return SCHED_OK;
     }
     if (h->batch_handle) return SCHED_E_INVAL;

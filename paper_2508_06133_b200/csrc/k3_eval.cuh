@@ -8,8 +8,8 @@
 //                     bucketed by first moved position); simulation resumes from the last snapshot
 //                     at or before the first moved position.
 //   k3_eval_orders    explicit permutations, simulated from t = 0.
-//   k3_eval_policy    one single-warp CTA per (instance, policy) pair: sort, optional prefix-F
-//                     batching, simulation -- all in shared memory.
+//   (k3_policy.cuh)   k3_eval_policy: one warp per (instance, policy) pair: order construction,
+//                     optional prefix-F batching, simulation -- all in shared memory.
 //   k3_check_starts   explicit start times: occupancy by the integer program's memory row
 //                     (Section 6.1), flag raised at the first round above M.
 //
@@ -258,139 +258,6 @@ k3_eval_orders(const OrderEvalParams p) {
         }
     }
     if (lane == 0) p.tel_out[c] = sim.total();
-}
-
-// ------------------------------------------------------------------------------------------------
-// Policy sweep: grid = B * P single-warp CTAs; CTA (b, k) evaluates instance b under policies[k].
-// Dynamic shared memory: the simulator's ring (SIM::ring_cells(L) ints); PT P[n+2], O[n+2] (PT =
-// int32 when n * M < 2^31, else int64); int s[n], o[n], boff[n+2]; 16-bit: three id buffers [n] and
-// batch numbers [n].  Orders are built by
-// a single-warp radix sort (k3_warp_radix_sort) on the fields of the policy's key.
-// ------------------------------------------------------------------------------------------------
-// One pass of a stable least-significant-digit radix sort run by a single warp on shared memory:
-// the m ids of `in` are written to `out` in ascending order of digit(id), an 8-bit value; ids with
-// equal digits keep their order.  `hist` is 256 ints of shared memory.  Every chunk of 32 ids is
-// ranked with a match-any vote (lanes with the same digit form a group whose lowest lane books the
-// group's bins), so no atomics are needed and the result does not depend on timing.
-template <class IT, class DIGIT>
-__device__ __forceinline__ void k3_warp_radix_pass(const IT* in, IT* out, int m, int* hist, int lane, DIGIT digit) {
-    for (int b = lane; b < 256; b += 32) hist[b] = 0;
-    __syncwarp();
-    const unsigned lt = (1u << lane) - 1u;
-    for (int e = lane; e < m; e += 32) atomicAdd(&hist[KV_IDX(digit(in[e]), 256, 901)], 1);   // count (order-free)
-    __syncwarp();
-    {                                                                // exclusive scan of the 256 bins, 8 per lane
-        int v[8], sum = 0;
-#pragma unroll
-        for (int k = 0; k < 8; ++k) { v[k] = hist[8 * lane + k]; sum += v[k]; }
-        int incl = sum;
-        for (int dlt = 1; dlt < 32; dlt <<= 1) {
-            const int y = __shfl_up_sync(KV_FULL, incl, dlt);
-            if (lane >= dlt) incl += y;
-        }
-        int run = incl - sum;
-#pragma unroll
-        for (int k = 0; k < 8; ++k) { hist[8 * lane + k] = run; run += v[k]; }
-    }
-    __syncwarp();
-    for (int base = 0; base < m; base += 32) {                       // scatter
-        const int e = base + lane;
-        const int id = e < m ? in[e] : 0;
-        const int d = e < m ? digit(id) : 256 + lane;
-        const unsigned peers = __match_any_sync(KV_FULL, d);
-        int pos = 0;
-        if (e < m) pos = (int)KV_IDX(hist[KV_IDX(d, 256, 902)] + __popc(peers & lt), m, 903);
-        __syncwarp();
-        if (e < m) {
-            out[pos] = (IT)id;
-            if ((peers & lt) == 0) hist[d] += __popc(peers);
-        }
-        __syncwarp();
-    }
-}
-
-// The m ids of `a` stably re-ordered by ascending field(id) (`bytes` 8-bit digits, least significant
-// first).  a and b are two id buffers of m ints; returns the one that holds the result.
-template <class IT, class FIELD>
-__device__ __forceinline__ IT* k3_warp_radix_sort(IT* a, IT* b, int m, int* hist, int lane, FIELD field, int bytes) {
-    for (int k = 0; k < bytes; ++k) {
-        k3_warp_radix_pass(a, b, m, hist, lane, [&](int id) { return (field(id) >> (8 * k)) & 255; });
-        IT* x = a; a = b; b = x;
-    }
-    return a;
-}
-
-__host__ __device__ __forceinline__ int k3_bytes_of(unsigned v) { int b = 1; while (v >> (8 * b) && b < 4) ++b; return b; }
-
-typedef unsigned short k3_id_t;                     // request ids and list positions of the policy kernel (n < 65,536)
-
-template <class SIM, typename PT>
-__global__ void __launch_bounds__(32)
-k3_eval_policy(const int* __restrict__ s_all, const int* __restrict__ o_all, int n, int L, int M, int omax,
-               const int* __restrict__ policies, int num_policies,
-               i64* __restrict__ tel_out, int* __restrict__ starts_out, int* status) {
-    extern __shared__ __align__(128) unsigned char smem_raw[];
-    const int lane = threadIdx.x;
-    const int b = blockIdx.x / num_policies, kpol = blockIdx.x % num_policies;
-    const int policy = policies[kpol];
-    int* ring = (int*)smem_raw;                       // first: 16-byte aligned for the vector loads
-    PT* P = (PT*)(ring + SIM::ring_cells(L));         // a multiple of 4 ints: 8-byte aligned
-    PT* O = P + (n + 2);
-    int* s = (int*)(O + (n + 2));
-    int* o = s + n;
-    int* boff = o + n;                                // n + 2 batch offsets
-    k3_id_t* bufa = (k3_id_t*)(boff + n + 2);
-    k3_id_t* bufb = bufa + n;
-    k3_id_t* byo = bufb + n;                          // ids by ascending (o, id) (Sorted-F keeps them for its second sort)
-    k3_id_t* bat = byo + n;                           // batch number of every request (Sorted-F)
-    __shared__ i64 sh_warp[33];                       // one warp: k2_prefix_sums uses words 0 and 32
-    __shared__ i64 carry[2];
-    __shared__ u64 sh_best[2];                        // one warp: k2_select_batches needs no cross-warp words
-    __shared__ int hist[256];
-
-    for (int i = lane; i < n; i += 32) {
-        s[i] = s_all[(size_t)b * n + i];
-        o[i] = o_all[(size_t)b * n + i];
-        bufa[i] = (k3_id_t)i;
-    }
-    __syncwarp();
-    const int o_bytes = k3_bytes_of((unsigned)omax), t_bytes = k3_bytes_of((unsigned)M);
-    auto f_o = [&](int id) { return o[id]; };
-    auto f_t = [&](int id) { return s[id] + o[id]; };
-    k3_id_t* ord = bufa;                              // FCFS: the identity order
-    // every sort is a chain of stable passes from the identity order, so ties end in ascending id
-    if (policy == SCHED_POLICY_SOF) {
-        ord = k3_warp_radix_sort(bufa, bufb, n, hist, lane, f_o, o_bytes);
-    } else if (policy == SCHED_POLICY_TOTAL_SIZE) {
-        ord = k3_warp_radix_sort(bufa, bufb, n, hist, lane, f_t, t_bytes);
-    } else if (policy == SCHED_POLICY_SORTED_F) {
-        // ascending (s+o, o, id) = the (o, id) order re-sorted stably by s+o; F-metric batch boundaries;
-        // then every batch by ascending (o, id) = the (o, id) order re-sorted stably by batch number
-        ord = k3_warp_radix_sort(bufa, bufb, n, hist, lane, f_o, o_bytes);
-        for (int i = lane; i < n; i += 32) byo[i] = ord[i];
-        __syncwarp();
-        k3_id_t* other = ord == bufa ? bufb : bufa;
-        ord = k3_warp_radix_sort(ord, other, n, hist, lane, f_t, t_bytes);
-        k2_prefix_sums(s, o, ord, n, P, O, sh_warp, carry);
-        __syncwarp();
-        const int nb = k2_select_batches(P, O, n, (i64)M, boff, sh_best);
-        __syncwarp();
-        for (int bi = 0; bi < nb; ++bi)
-            for (int q = boff[bi] + lane; q < boff[bi + 1]; q += 32) bat[KV_IDX(ord[KV_IDX(q, n, 904)], n, 905)] = bi;
-        __syncwarp();
-        auto f_b = [&](int id) { return bat[id]; };
-        ord = k3_warp_radix_sort(byo, ord == bufa ? bufb : bufa, n, hist, lane, f_b, k3_bytes_of((unsigned)nb));
-    }
-    SIM sim;
-    sim.attach(ring, L);
-    sim.reset(lane);
-    int* starts = starts_out ? starts_out + ((size_t)b * num_policies + kpol) * n : nullptr;
-    for (int q = 0; q < n; ++q) {
-        const int id = (int)KV_IDX(ord[q], n, 906);
-        const int pstart = sim.admit(s[id], o[id], M, lane, status);
-        if (starts && lane == 0) starts[id] = pstart;
-    }
-    if (lane == 0) tel_out[(size_t)b * num_policies + kpol] = sim.total();
 }
 
 // ------------------------------------------------------------------------------------------------
